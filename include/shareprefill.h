@@ -1,0 +1,187 @@
+/*
+ * shareprefill.h - C ABI of the SharePrefill prefill-attention library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library computes the attention of ONE transformer layer during prefill
+ * the way SharePrefill (arXiv 2505.19578) does it, with the per-head pattern
+ * decision given by the caller:
+ *
+ *   1. "pivot" heads run exact dense causal attention and, in the same pass,
+ *      emit a block-importance map: the softmax probability mass of every
+ *      (query-block, key-block) tile                       [sp_dense_pivot_attn]
+ *   2. each row-block of the map is reduced to a block mask by a cumulative
+ *      mass threshold gamma (Algorithm "Construct Pivotal Pattern")
+ *                                                [sp_block_mask_from_importance]
+ *   3. the mask is shared with every head of the pivot's cluster (Algorithm
+ *      "Share Pivotal Pattern"), and those heads run block-sparse causal
+ *      attention over the selected tiles only (Section 5.1, masked attention
+ *      A(Q,K,V,M))                                         [sp_block_sparse_attn]
+ *
+ *   sp_prefill_attn chains 1-3 on one stream.
+ *
+ * General conventions
+ *   - Every function returns an int: SP_OK (0) or a negative SP_ERR_* code.
+ *     Nothing throws, prints or exits.
+ *   - Pointers are DEVICE pointers unless the comment says "host".
+ *   - Calls validate on the host, enqueue kernels on `stream` (a cudaStream_t
+ *     passed as void*; NULL = the default stream) and return WITHOUT
+ *     synchronising.  Errors detected on the device (a bounded wait that ran
+ *     out) are reported by sp_get_status after the caller has synchronised.
+ *   - The caller owns every tensor and the stream.  The library owns only the
+ *     sp_ctx (its workspace and status word).  A context belongs to one device
+ *     and must not be used from two streams at the same time.
+ *   - Tensors are bf16, logical shape [batch, heads, seq, head_dim], element
+ *     strides given explicitly; stride[3] must be 1 and the other strides must
+ *     be multiples of 8 elements (16 bytes); data must be 16-byte aligned.
+ *     batch must be 1.
+ *   - Supported: head_dim in {64, 128}; block in {64, 128}; seq a multiple of
+ *     block; n_q_heads a multiple of n_kv_heads; seq / block <= 1024.
+ *     Anything else returns SP_ERR_UNSUPPORTED.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - Nb = seq / block.  Row-block i = query rows [i*block, (i+1)*block);
+ *     key-block j likewise.  Attention is causal: key c is visible to query r
+ *     iff c <= r, so only tiles j <= i exist.
+ */
+#ifndef SHAREPREFILL_H_
+#define SHAREPREFILL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  SP_OK = 0,
+  SP_ERR_INVALID_ARG = -1, /* NULL pointer, bad shape/stride, gamma not in (0, +inf), ... */
+  SP_ERR_UNSUPPORTED = -2, /* a size outside the supported set listed above            */
+  SP_ERR_WORKSPACE = -3,   /* workspace allocation failed                              */
+  SP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                      */
+  SP_ERR_TIMEOUT = -5      /* a bounded device-side wait ran out (see sp_get_status)   */
+};
+
+/* bf16 tensor view: device pointer, sizes and strides in ELEMENTS. */
+typedef struct {
+  void* data;
+  int64_t shape[4];  /* [batch, heads, seq, head_dim] */
+  int64_t stride[4]; /* stride[3] == 1                 */
+} sp_tensor;
+
+typedef struct sp_ctx sp_ctx;
+
+/* Create / destroy a context on CUDA device `device`.  Creation allocates a
+ * small status buffer; the workspace grows on demand (cudaMalloc, which
+ * synchronises the device) or ahead of time with sp_ctx_reserve. */
+int sp_ctx_create(sp_ctx** out, int device);
+int sp_ctx_destroy(sp_ctx* ctx);
+
+/* Bytes of workspace sp_prefill_attn needs for a problem of this size
+ * (importance maps, masks, compacted lists, per-tile softmax statistics). */
+int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block,
+                       int n_pivots, size_t* bytes /* host, out */);
+
+/* Make sure the context's workspace holds at least `bytes`. */
+int sp_ctx_reserve(sp_ctx* ctx, size_t bytes);
+
+/* Read and clear the device status word.  The caller must have synchronised
+ * the stream(s) it used.  *code is SP_OK or SP_ERR_TIMEOUT; *where identifies
+ * the wait that gave up (kernel-internal id).  Either pointer may be NULL. */
+int sp_get_status(sp_ctx* ctx, int* code /* host, out */, int* where /* host, out */);
+
+/* Static string for an SP_* code. */
+const char* sp_strerror(int code);
+
+/*
+ * Step 1 - dense causal attention of selected heads, with block importance.
+ *   (Algorithm "Share Pivotal Pattern": a head without a pivotal pattern gets
+ *   the all-ones pattern and computes full attention; Section 5.2, "Sparse
+ *   Attention Computation": the kernel emits a per-block statistic in the same
+ *   pass that produces the output.)
+ *
+ *   heads           host, [n_heads]: query-head indices to process.
+ *   out             same shape as q; rows of the listed heads are overwritten.
+ *   importance_out  device fp32 [n_heads, Nb, Nb], or NULL for plain dense
+ *                   attention.  Entry [t][i][j] = (1/block) * sum over rows r of
+ *                   row-block i and keys c of key-block j (c <= r) of the softmax
+ *                   probability P[r][c] of head heads[t]; each row-block's entries
+ *                   sum to 1; entries with j > i are written as 0.
+ *   lse_out         device fp32 [n_heads, seq] natural-log-sum-exp of the scaled
+ *                   logits of each query row, or NULL.
+ */
+int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                        const int32_t* heads, int n_heads, int block, sp_tensor* out,
+                        float* importance_out, float* lse_out, void* stream);
+
+/*
+ * Step 2 - importance map -> block mask and compacted key-block lists.
+ *   (Algorithm "Construct Pivotal Pattern": sort the scores, take the minimum
+ *   budget K whose top-K sum reaches gamma, turn the index set into a mask.)
+ *   Each row-block i of each of the `n_maps` maps is treated independently over
+ *   its causal entries j = 0..i: order by importance descending (equal values:
+ *   smaller j first), running sum in that order in float64, K_i = first k whose
+ *   sum >= gamma (all i+1 entries if the sum never gets there); the first K_i
+ *   entries of the order are selected.
+ *
+ *   importance   device fp32 [n_maps, nb, nb]; entries must be finite and >= 0
+ *                (anything else is read as 0); entries with j > i are ignored.
+ *   gamma        > 0.  Compared as the double nearest to this float.
+ *   mask_out     device u8  [n_maps, nb, nb]: 1 = compute, 0 = skip (j > i: 0); may be NULL.
+ *   counts_out   device i32 [n_maps, nb]: K_i.
+ *   indices_out  device i32 [n_maps, nb, nb]: row i holds the K_i selected
+ *                key-blocks in ascending order, then -1 up to nb.
+ */
+int sp_block_mask_from_importance(sp_ctx* ctx, const float* importance, int n_maps, int nb,
+                                  float gamma, uint8_t* mask_out, int32_t* counts_out,
+                                  int32_t* indices_out, void* stream);
+
+/*
+ * Step 3 - block-sparse causal attention (Section 5.1: A(Q,K,V,M) =
+ *   softmax(QK^T/sqrt(d) - c(1-M)) V with c -> infinity, causal).
+ *
+ *   heads         host, [n_heads]: query heads to process.
+ *   list_of_head  host, [n_heads]: which list (first index of counts/indices)
+ *                 each listed head walks; -1 = all causal tiles (dense).
+ *   counts        device i32 [n_lists, nb]; indices device i32 [n_lists, nb, nb]
+ *                 as written by sp_block_mask_from_importance.  Every listed
+ *                 row must select at least one key-block and only j <= i.
+ *   out           rows of the listed heads are overwritten.
+ */
+int sp_block_sparse_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                         const int32_t* heads, int n_heads, const int32_t* list_of_head,
+                         const int32_t* counts, const int32_t* indices, int n_lists, int block,
+                         sp_tensor* out, void* stream);
+
+/*
+ * The whole layer (Algorithm "Sparse Attention" with the pattern decision fixed
+ * by the caller): pivots dense + importance, importance -> mask, members sparse.
+ *
+ *   cluster_map  host, [n_q_heads]: cluster id of each query head; < 0 = no cluster.
+ *   pivot_heads  host, [n_pivots]: heads that run dense and construct a pattern.
+ *                The pivot of a cluster is the FIRST listed pivot head belonging
+ *                to it.  A non-pivot head whose cluster has no pivot (or whose
+ *                id is < 0) runs dense.
+ *   gamma, block as above.
+ *   out          bf16, same shape as q; fully overwritten.
+ *   mask_out     device u8 [n_q_heads, Nb, Nb] or NULL: the pattern of each head:
+ *                for a member its cluster pivot's mask, for a pivot the mask it
+ *                constructed (its own output is dense), for a head that ran dense
+ *                without constructing anything the causal all-ones mask.
+ */
+int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                    const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
+                    float gamma, int block, sp_tensor* out, uint8_t* mask_out, void* stream);
+
+/* Which attention kernel the context launches: 0 = tensor-core kernel
+ * (tcgen05 / TMEM / TMA; the product path, default), 1 = plain fp32 CUDA-core
+ * kernel kept as an independent on-device cross-check. */
+int sp_ctx_set_kernel(sp_ctx* ctx, int which);
+
+/* Number of kernels this context has launched since creation (for callers
+ * that account for launches). */
+int64_t sp_ctx_launch_count(const sp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SHAREPREFILL_H_ */

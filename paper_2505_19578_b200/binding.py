@@ -1,0 +1,186 @@
+"""Thin ctypes binding over libshareprefill.so (see include/shareprefill.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch is used for device memory and streams.  There is no fallback:
+if the shared library has not been built, loading raises.
+
+Tensors: q [Hq, N, d] or [1, Hq, N, d] bf16 CUDA; k, v [Hkv, N, d] likewise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libshareprefill.so")
+
+SP_OK = 0
+SP_ERR_INVALID_ARG = -1
+SP_ERR_UNSUPPORTED = -2
+SP_ERR_WORKSPACE = -3
+SP_ERR_CUDA = -4
+SP_ERR_TIMEOUT = -5
+
+EXPORTS = (
+    "sp_ctx_create", "sp_ctx_destroy", "sp_workspace_bytes", "sp_ctx_reserve", "sp_get_status",
+    "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
+    "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count",
+)
+
+
+class SpTensor(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4)]
+
+
+class SpError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {error_string(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the shared library; raises if it is missing (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2505_19578_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P, I, F = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    T = ctypes.POINTER(SpTensor)
+    IP = ctypes.POINTER(ctypes.c_int32)
+    lib.sp_ctx_create.argtypes = [ctypes.POINTER(P), I]
+    lib.sp_ctx_destroy.argtypes = [P]
+    lib.sp_workspace_bytes.argtypes = [ctypes.c_int64, I, I, I, I, I, ctypes.POINTER(ctypes.c_size_t)]
+    lib.sp_ctx_reserve.argtypes = [P, ctypes.c_size_t]
+    lib.sp_get_status.argtypes = [P, ctypes.POINTER(I), ctypes.POINTER(I)]
+    lib.sp_strerror.argtypes = [I]
+    lib.sp_strerror.restype = ctypes.c_char_p
+    lib.sp_dense_pivot_attn.argtypes = [P, T, T, T, IP, I, I, T, P, P, P]
+    lib.sp_block_mask_from_importance.argtypes = [P, P, I, I, F, P, P, P, P]
+    lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
+    lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
+    lib.sp_ctx_set_kernel.argtypes = [P, I]
+    lib.sp_ctx_launch_count.argtypes = [P]
+    lib.sp_ctx_launch_count.restype = ctypes.c_int64
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if name not in ("sp_strerror", "sp_ctx_launch_count"):
+            fn.restype = I
+    _lib = lib
+    return lib
+
+
+def error_string(code: int) -> str:
+    return load().sp_strerror(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != SP_OK:
+        raise SpError(code, what)
+
+
+def _view(t: torch.Tensor) -> SpTensor:
+    if t.dim() == 3:
+        t = t.unsqueeze(0)
+    if t.dim() != 4 or t.dtype != torch.bfloat16 or not t.is_cuda:
+        raise ValueError("expected a CUDA bf16 tensor [heads, seq, dim] or [1, heads, seq, dim]")
+    s = SpTensor()
+    s.data = t.data_ptr()
+    for x in range(4):
+        s.shape[x] = t.shape[x]
+        # the stride of a size-1 dimension is never used; report 0 for it
+        s.stride[x] = t.stride(x) if (t.shape[x] > 1 or x == 3) else 0
+    return s
+
+
+def _i32(xs):
+    xs = list(xs)
+    return (ctypes.c_int32 * max(len(xs), 1))(*xs)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Context:
+    """Owns one sp_ctx (workspace + status word) on one CUDA device."""
+
+    def __init__(self, device: int | None = None, kernel: str = "tc"):
+        self._lib = load()
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        h = ctypes.c_void_p()
+        _check(self._lib.sp_ctx_create(ctypes.byref(h), self.device), "sp_ctx_create")
+        self._h = h
+        self.set_kernel(kernel)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.sp_ctx_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def set_kernel(self, kernel: str):
+        _check(self._lib.sp_ctx_set_kernel(self._h, {"tc": 0, "simt": 1}[kernel]), "sp_ctx_set_kernel")
+
+    def launch_count(self) -> int:
+        return int(self._lib.sp_ctx_launch_count(self._h))
+
+    def reserve(self, nbytes: int):
+        _check(self._lib.sp_ctx_reserve(self._h, nbytes), "sp_ctx_reserve")
+
+    def status(self):
+        """(code, where) of the device status word; call after synchronising."""
+        c, w = ctypes.c_int(), ctypes.c_int()
+        _check(self._lib.sp_get_status(self._h, ctypes.byref(c), ctypes.byref(w)), "sp_get_status")
+        return c.value, w.value
+
+    # ---- the four calls -------------------------------------------------
+
+    def sp_dense_pivot_attn(self, q, k, v, heads, block, out, importance_out=None, lse_out=None, stream=None):
+        heads = list(heads)
+        _check(self._lib.sp_dense_pivot_attn(self._h, _view(q), _view(k), _view(v), _i32(heads), len(heads), block,
+                                             _view(out), _ptr(importance_out), _ptr(lse_out), _stream(stream)),
+               "sp_dense_pivot_attn")
+
+    def sp_block_mask_from_importance(self, importance, gamma, mask_out, counts_out, indices_out, stream=None):
+        n_maps, nb, nb2 = importance.shape
+        assert nb == nb2 and importance.dtype == torch.float32 and importance.is_contiguous()
+        _check(self._lib.sp_block_mask_from_importance(self._h, _ptr(importance), n_maps, nb, gamma, _ptr(mask_out),
+                                                       _ptr(counts_out), _ptr(indices_out), _stream(stream)),
+               "sp_block_mask_from_importance")
+
+    def sp_block_sparse_attn(self, q, k, v, heads, list_of_head, counts, indices, block, out, stream=None):
+        heads, list_of_head = list(heads), list(list_of_head)
+        assert len(heads) == len(list_of_head)
+        n_lists = 0 if counts is None else counts.shape[0]
+        _check(self._lib.sp_block_sparse_attn(self._h, _view(q), _view(k), _view(v), _i32(heads), len(heads),
+                                              _i32(list_of_head), _ptr(counts), _ptr(indices), n_lists, block,
+                                              _view(out), _stream(stream)),
+               "sp_block_sparse_attn")
+
+    def sp_prefill_attn(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
+        cluster_map, pivot_heads = list(cluster_map), list(pivot_heads)
+        _check(self._lib.sp_prefill_attn(self._h, _view(q), _view(k), _view(v), _i32(cluster_map), _i32(pivot_heads),
+                                         len(pivot_heads), gamma, block, _view(out), _ptr(mask_out), _stream(stream)),
+               "sp_prefill_attn")
+
+
+def workspace_bytes(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots) -> int:
+    out = ctypes.c_size_t()
+    _check(load().sp_workspace_bytes(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots, ctypes.byref(out)),
+           "sp_workspace_bytes")
+    return out.value

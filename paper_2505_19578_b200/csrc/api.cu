@@ -1,0 +1,377 @@
+// Host side of the C ABI: argument validation, workspace carving, the sharing
+// table (Algorithm "Share Pivotal Pattern") and the launch sequence of
+// sp_prefill_attn (Algorithm "Sparse Attention" with the pattern decision fixed
+// by the caller).  No arithmetic of the method happens on the host.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+struct sp_ctx {
+  int device = 0;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int* status = nullptr;  // device int[2]
+  int kernel = 0;         // 0 tensor-core, 1 CUDA-core cross-check
+  int64_t launches = 0;
+};
+
+namespace {
+
+using namespace sp;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    target = dev;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0 && prev != target) cudaSetDevice(prev);
+  }
+  int target = -1;
+};
+
+size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Problem {
+  int Hq, Hkv, N, d, B, Nb;
+};
+
+int check_tensor(const sp_tensor* t) {
+  if (!t || !t->data) return SP_ERR_INVALID_ARG;
+  for (int x = 0; x < 4; ++x)
+    if (t->shape[x] <= 0) return SP_ERR_INVALID_ARG;
+  if (t->stride[3] != 1) return SP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(t->data) & 15) != 0) return SP_ERR_INVALID_ARG;
+  for (int x = 0; x < 3; ++x)
+    if (t->stride[x] < 0 || (t->stride[x] % 8) != 0) return SP_ERR_INVALID_ARG;
+  if (t->stride[2] < t->shape[3]) return SP_ERR_INVALID_ARG;
+  return SP_OK;
+}
+
+int check_problem(const sp_tensor* q, const sp_tensor* k, const sp_tensor* v, const sp_tensor* out, int block,
+                  Problem* p) {
+  int rc;
+  if ((rc = check_tensor(q)) || (rc = check_tensor(k)) || (rc = check_tensor(v)) || (rc = check_tensor(out))) return rc;
+  for (int x = 0; x < 4; ++x) {
+    if (k->shape[x] != v->shape[x]) return SP_ERR_INVALID_ARG;
+    if (q->shape[x] != out->shape[x]) return SP_ERR_INVALID_ARG;
+  }
+  if (q->shape[2] != k->shape[2] || q->shape[3] != k->shape[3]) return SP_ERR_INVALID_ARG;
+  if (q->shape[0] != k->shape[0]) return SP_ERR_INVALID_ARG;
+  if (q->shape[0] != 1) return SP_ERR_UNSUPPORTED;
+  const int64_t Hq = q->shape[1], Hkv = k->shape[1], N = q->shape[2], d = q->shape[3];
+  if (Hq > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  if (Hq % Hkv != 0) return SP_ERR_UNSUPPORTED;
+  if (d != 64 && d != 128) return SP_ERR_UNSUPPORTED;
+  if (block != 64 && block != 128) return SP_ERR_UNSUPPORTED;
+  if (N % block != 0) return SP_ERR_UNSUPPORTED;
+  if (N / block > kMaxNb) return SP_ERR_UNSUPPORTED;
+  p->Hq = (int)Hq; p->Hkv = (int)Hkv; p->N = (int)N; p->d = (int)d; p->B = block; p->Nb = (int)(N / block);
+  return SP_OK;
+}
+
+AttnArgs base_args(const sp_ctx* ctx, const Problem& p, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                   const sp_tensor* out) {
+  AttnArgs a;
+  memset(&a, 0, sizeof(a));
+  a.q = static_cast<const __nv_bfloat16*>(q->data);
+  a.k = static_cast<const __nv_bfloat16*>(k->data);
+  a.v = static_cast<const __nv_bfloat16*>(v->data);
+  a.o = static_cast<__nv_bfloat16*>(out->data);
+  a.q_sh = q->stride[1]; a.q_sn = q->stride[2];
+  a.k_sh = k->stride[1]; a.k_sn = k->stride[2];
+  a.v_sh = v->stride[1]; a.v_sn = v->stride[2];
+  a.o_sh = out->stride[1]; a.o_sn = out->stride[2];
+  a.n_q_heads = p.Hq; a.n_kv_heads = p.Hkv;
+  a.N = p.N; a.d = p.d; a.B = p.B; a.Nb = p.Nb; a.group = p.Hq / p.Hkv;
+  a.status = ctx->status;
+  a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.d));
+  return a;
+}
+
+int reserve(sp_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->ws_bytes) return SP_OK;
+  if (ctx->ws) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return SP_ERR_CUDA;
+    cudaFree(ctx->ws);
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+  }
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return SP_ERR_WORKSPACE;
+  }
+  ctx->ws = p;
+  ctx->ws_bytes = bytes;
+  return SP_OK;
+}
+
+int launch_attn(sp_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
+  if (a.n_heads == 0) return SP_OK;
+  cudaError_t e = ctx->kernel == 1 ? launch_attn_simt(a, s) : launch_attn_tc(a, s);
+  if (e != cudaSuccess) return SP_ERR_CUDA;
+  ctx->launches += 1;
+  return SP_OK;
+}
+
+struct WsLayout {
+  size_t imp, mask, counts, indices, stats, total;
+};
+
+WsLayout ws_layout(int Nb, int B, int n_pivots) {
+  WsLayout w;
+  size_t off = 0;
+  const size_t nn = (size_t)Nb * Nb;
+  w.imp = off;     off += align_up(n_pivots * nn * sizeof(float));
+  w.mask = off;    off += align_up(n_pivots * nn);
+  w.counts = off;  off += align_up((size_t)n_pivots * Nb * sizeof(int32_t));
+  w.indices = off; off += align_up(n_pivots * nn * sizeof(int32_t));
+  w.stats = off;   off += align_up(n_pivots * tile_stats_bytes_per_head(Nb, B));
+  w.total = off;
+  return w;
+}
+
+__global__ void gather_masks_kernel(const uint8_t* __restrict__ pivot_masks, HeadTable src, int nb,
+                                    uint8_t* __restrict__ out) {
+  const int i = blockIdx.x, h = blockIdx.y;
+  const int s = src.v[h];
+  uint8_t* dst = out + ((size_t)h * nb + i) * nb;
+  if (s >= 0) {
+    const uint8_t* from = pivot_masks + ((size_t)s * nb + i) * nb;
+    for (int j = threadIdx.x; j < nb; j += blockDim.x) dst[j] = from[j];
+  } else {
+    for (int j = threadIdx.x; j < nb; j += blockDim.x) dst[j] = j <= i ? 1 : 0;
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sp_strerror(int code) {
+  switch (code) {
+    case SP_OK: return "ok";
+    case SP_ERR_INVALID_ARG: return "invalid argument";
+    case SP_ERR_UNSUPPORTED: return "unsupported size or layout";
+    case SP_ERR_WORKSPACE: return "workspace allocation failed";
+    case SP_ERR_CUDA: return "CUDA call failed";
+    case SP_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown error code";
+  }
+}
+
+int sp_ctx_create(sp_ctx** out, int device) {
+  if (!out) return SP_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess) { cudaGetLastError(); return SP_ERR_CUDA; }
+  if (device < 0 || device >= n) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(device);
+  if (!g.ok) return SP_ERR_CUDA;
+  sp_ctx* c = new (std::nothrow) sp_ctx();
+  if (!c) return SP_ERR_WORKSPACE;
+  c->device = device;
+  if (cudaMalloc(&c->status, 2 * sizeof(int)) != cudaSuccess || cudaMemset(c->status, 0, 2 * sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    delete c;
+    return SP_ERR_CUDA;
+  }
+  *out = c;
+  return SP_OK;
+}
+
+int sp_ctx_destroy(sp_ctx* ctx) {
+  if (!ctx) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->status) cudaFree(ctx->status);
+  delete ctx;
+  return SP_OK;
+}
+
+int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block, int n_pivots,
+                       size_t* bytes) {
+  if (!bytes || seq <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_pivots < 0) return SP_ERR_INVALID_ARG;
+  if (block != 64 && block != 128) return SP_ERR_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return SP_ERR_UNSUPPORTED;
+  if (seq % block != 0 || seq / block > kMaxNb || n_q_heads % n_kv_heads != 0) return SP_ERR_UNSUPPORTED;
+  *bytes = ws_layout((int)(seq / block), block, n_pivots).total;
+  return SP_OK;
+}
+
+int sp_ctx_reserve(sp_ctx* ctx, size_t bytes) {
+  if (!ctx) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  return reserve(ctx, bytes);
+}
+
+int sp_get_status(sp_ctx* ctx, int* code, int* where) {
+  if (!ctx) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  int host[2] = {0, 0};
+  if (cudaMemcpy(host, ctx->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return SP_ERR_CUDA;
+  if (host[0] != 0 && cudaMemset(ctx->status, 0, sizeof(host)) != cudaSuccess) return SP_ERR_CUDA;
+  if (code) *code = host[0];
+  if (where) *where = host[1];
+  return SP_OK;
+}
+
+int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
+  if (!ctx || (which != 0 && which != 1)) return SP_ERR_INVALID_ARG;
+  ctx->kernel = which;
+  return SP_OK;
+}
+
+int64_t sp_ctx_launch_count(const sp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v, const int32_t* heads,
+                        int n_heads, int block, sp_tensor* out, float* importance_out, float* lse_out, void* stream) {
+  if (!ctx || !heads || n_heads < 0) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  for (int t = 0; t < n_heads; ++t)
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  AttnArgs a = base_args(ctx, p, q, k, v, out);
+  a.n_heads = n_heads;
+  for (int t = 0; t < n_heads; ++t) { a.heads.v[t] = heads[t]; a.lists.v[t] = -1; }
+  a.importance = importance_out;
+  a.lse = lse_out;
+  if (importance_out && ctx->kernel == 0) {
+    if ((rc = reserve(ctx, align_up((size_t)n_heads * tile_stats_bytes_per_head(p.Nb, p.B))))) return rc;
+    a.tile_stats = static_cast<float*>(ctx->ws);
+  }
+  return launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+int sp_block_mask_from_importance(sp_ctx* ctx, const float* importance, int n_maps, int nb, float gamma,
+                                  uint8_t* mask_out, int32_t* counts_out, int32_t* indices_out, void* stream) {
+  if (!ctx || !importance || !counts_out || !indices_out || n_maps < 0 || nb <= 0) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  if (nb > kMaxNb) return SP_ERR_UNSUPPORTED;
+  if (n_maps == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  MaskArgs m{importance, n_maps, nb, (double)gamma, mask_out, counts_out, indices_out};
+  if (launch_block_mask(m, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  ctx->launches += 1;
+  return SP_OK;
+}
+
+int sp_block_sparse_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v, const int32_t* heads,
+                         int n_heads, const int32_t* list_of_head, const int32_t* counts, const int32_t* indices,
+                         int n_lists, int block, sp_tensor* out, void* stream) {
+  if (!ctx || !heads || !list_of_head || n_heads < 0 || n_lists < 0) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  bool any_list = false;
+  for (int t = 0; t < n_heads; ++t) {
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+    if (list_of_head[t] >= n_lists) return SP_ERR_INVALID_ARG;
+    any_list |= list_of_head[t] >= 0;
+  }
+  if (any_list && (!counts || !indices)) return SP_ERR_INVALID_ARG;
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  AttnArgs a = base_args(ctx, p, q, k, v, out);
+  a.n_heads = n_heads;
+  for (int t = 0; t < n_heads; ++t) { a.heads.v[t] = heads[t]; a.lists.v[t] = list_of_head[t] < 0 ? -1 : list_of_head[t]; }
+  a.counts = counts;
+  a.indices = indices;
+  return launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                    const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots, float gamma, int block,
+                    sp_tensor* out, uint8_t* mask_out, void* stream) {
+  if (!ctx || !cluster_map || n_pivots < 0 || (n_pivots > 0 && !pivot_heads)) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (n_pivots > p.Hq) return SP_ERR_INVALID_ARG;
+
+  // Sharing table: pivot slot of each cluster = first listed pivot belonging to it.
+  int pivot_slot_of_head[kMaxHeads];
+  for (int h = 0; h < p.Hq; ++h) pivot_slot_of_head[h] = -1;
+  for (int t = 0; t < n_pivots; ++t) {
+    const int h = pivot_heads[t];
+    if (h < 0 || h >= p.Hq || pivot_slot_of_head[h] >= 0) return SP_ERR_INVALID_ARG;  // range / duplicate
+    pivot_slot_of_head[h] = t;
+  }
+  auto cluster_pivot = [&](int c) {
+    if (c < 0) return -1;
+    for (int t = 0; t < n_pivots; ++t)
+      if (cluster_map[pivot_heads[t]] == c) return t;
+    return -1;
+  };
+
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots);
+  if ((rc = reserve(ctx, w.total))) return rc;
+  char* ws = static_cast<char*>(ctx->ws);
+  float* imp = reinterpret_cast<float*>(ws + w.imp);
+  uint8_t* pmask = reinterpret_cast<uint8_t*>(ws + w.mask);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + w.counts);
+  int32_t* indices = reinterpret_cast<int32_t*>(ws + w.indices);
+  float* stats = reinterpret_cast<float*>(ws + w.stats);
+
+  // 1. pivots: dense + importance
+  AttnArgs a = base_args(ctx, p, q, k, v, out);
+  a.n_heads = n_pivots;
+  for (int t = 0; t < n_pivots; ++t) { a.heads.v[t] = pivot_heads[t]; a.lists.v[t] = -1; }
+  a.importance = imp;
+  a.tile_stats = stats;
+  if ((rc = launch_attn(ctx, a, s))) return rc;
+
+  // 2. importance -> masks and lists
+  if (n_pivots > 0) {
+    MaskArgs m{imp, n_pivots, p.Nb, (double)gamma, pmask, counts, indices};
+    if (launch_block_mask(m, s) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+  }
+
+  // 3. everyone else: the cluster pivot's list, or dense when there is none
+  AttnArgs b = base_args(ctx, p, q, k, v, out);
+  b.counts = counts;
+  b.indices = indices;
+  HeadTable mask_src;
+  int nb_heads = 0;
+  for (int h = 0; h < p.Hq; ++h) {
+    if (pivot_slot_of_head[h] >= 0) { mask_src.v[h] = pivot_slot_of_head[h]; continue; }
+    const int t = cluster_pivot(cluster_map[h]);
+    mask_src.v[h] = t;
+    b.heads.v[nb_heads] = h;
+    b.lists.v[nb_heads] = t;
+    ++nb_heads;
+  }
+  b.n_heads = nb_heads;
+  if ((rc = launch_attn(ctx, b, s))) return rc;
+
+  if (mask_out) {
+    gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, s>>>(pmask, mask_src, p.Nb, mask_out);
+    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+  }
+  return SP_OK;
+}
+
+}  // extern "C"

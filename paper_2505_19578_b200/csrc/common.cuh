@@ -1,0 +1,61 @@
+// Internal declarations shared by the library's translation units.
+// Nothing here is part of the C ABI (see include/shareprefill.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "shareprefill.h"
+
+namespace sp {
+
+constexpr int kMaxHeads = 128;   // query heads per call (kernel-parameter tables)
+constexpr int kMaxNb = 1024;     // key-blocks per row (mask kernel sorts one row per warp)
+
+struct HeadTable {
+  int32_t v[kMaxHeads];
+};
+
+// Everything an attention launch needs.  Strides are in elements.
+struct AttnArgs {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  __nv_bfloat16* o;
+  int64_t q_sh, q_sn, k_sh, k_sn, v_sh, v_sn, o_sh, o_sn;
+  int n_q_heads, n_kv_heads;
+  int N, d, B, Nb, group;  // group = n_q_heads / n_kv_heads
+  int n_heads;             // heads processed by this launch
+  HeadTable heads;         // query-head index per slot
+  HeadTable lists;         // list index per slot, -1 = dense (all causal tiles)
+  const int32_t* counts;   // [n_lists, Nb]       (may be null when every slot is dense)
+  const int32_t* indices;  // [n_lists, Nb, Nb]
+  float* importance;       // [n_heads, Nb, Nb] or null
+  float* lse;              // [n_heads, N] or null
+  float* tile_stats;       // scratch: per (slot, row-block) B floats per causal tile (tensor-core path)
+  int* status;             // device int[2]: {code, where}
+  float scale_log2;        // log2(e) / sqrt(d)
+};
+
+struct MaskArgs {
+  const float* importance;
+  int n_maps, nb;
+  double gamma;
+  uint8_t* mask;
+  int32_t* counts;
+  int32_t* indices;
+};
+
+// kernel launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA
+cudaError_t launch_block_mask(const MaskArgs& a, cudaStream_t s);
+cudaError_t launch_fill_causal_mask(uint8_t* mask, int nb, cudaStream_t s);
+
+// bytes of per-tile softmax statistics the tensor-core kernel spills for one head
+inline size_t tile_stats_bytes_per_head(int Nb, int B) {
+  return (size_t)Nb * (size_t)(Nb + 1) / 2 * (size_t)B * sizeof(float);
+}
+
+}  // namespace sp

@@ -50,13 +50,13 @@ class LayerConfig:
 
 CONFIGS = {
     # tiny parity config
-    "tiny": LayerConfig("tiny", 2048, 8, 8, 64, 64, 1e4, 16, 2, (0.3, 0.3), 10.0),
+    "tiny": LayerConfig("tiny", 2048, 8, 8, 64, 64, 1e4, 16, 2, (0.3, 0.3), 10.5),
     # Llama-3-8B-shaped layer, 32K
-    "llama8b_32k": LayerConfig("llama8b_32k", 32768, 32, 8, 128, 128, 5e5, 64, 8, (0.3, 0.3), 12.0),
+    "llama8b_32k": LayerConfig("llama8b_32k", 32768, 32, 8, 128, 128, 5e5, 64, 8, (0.3, 0.3), 12.5),
     # Llama-3-8B-shaped layer, 128K, 4 pivots per 32 heads
-    "llama8b_128k": LayerConfig("llama8b_128k", 131072, 32, 8, 128, 128, 5e5, 256, 4, (0.3, 0.3), 13.0),
+    "llama8b_128k": LayerConfig("llama8b_128k", 131072, 32, 8, 128, 128, 5e5, 256, 4, (0.3, 0.3), 13.5),
     # Qwen2.5-7B-shaped layer, 64K, GQA 7
-    "qwen7b_64k": LayerConfig("qwen7b_64k", 65536, 28, 4, 128, 128, 1e6, 64, 7, (0.2, 0.6), 12.5),
+    "qwen7b_64k": LayerConfig("qwen7b_64k", 65536, 28, 4, 128, 128, 1e6, 64, 7, (0.2, 0.6), 13.0),
 }
 
 

@@ -1,0 +1,59 @@
+"""The C-ABI library builds, loads without a GPU, and exports every symbol
+that include/shareprefill.h declares.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2505_19578_b200 import binding, build
+    build.build()
+    return binding.load()
+
+
+def _declared():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            txt = open(os.path.join(inc, f)).read()
+            txt = re.sub(r"/\*.*?\*/", "", txt, flags=re.S)
+            names |= set(re.findall(r"\b(sp_[a-z0-9_]+)\s*\(", txt))
+    return names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2505_19578_b200 import binding
+    names = _declared()
+    assert {"sp_prefill_attn", "sp_dense_pivot_attn", "sp_block_mask_from_importance",
+            "sp_block_sparse_attn"} <= names
+    assert names == set(binding.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_host_only_calls(lib):
+    from paper_2505_19578_b200 import binding
+    assert binding.error_string(0) == "ok"
+    assert "timed out" in binding.error_string(binding.SP_ERR_TIMEOUT)
+    b = binding.workspace_bytes(131072, 32, 8, 128, 128, 4)
+    nb = 1024
+    # importance + mask + counts + lists + per-tile statistics
+    assert b >= 4 * nb * nb * (4 + 1 + 4) + 4 * nb * (nb + 1) // 2 * 128 * 4
+    out = ctypes.c_size_t()
+    assert lib.sp_workspace_bytes(1000, 32, 8, 128, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED
+    assert lib.sp_workspace_bytes(4096, 32, 8, 96, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED
+    assert lib.sp_workspace_bytes(4096, 32, 8, 128, 128, 4, None) == binding.SP_ERR_INVALID_ARG
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    from paper_2505_19578_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load()

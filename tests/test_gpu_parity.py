@@ -1,0 +1,312 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64
+oracle on the same seeded bf16 inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import shareprefill_oracle as orc
+from paper_2505_19578_b200 import synth
+from tests import _parity as par
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = ["tc", "simt"]
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2505_19578_b200 import binding as b, build
+    build.build()
+    return b
+
+
+def _rand_layer(seed, Hq, Hkv, N, d, scale=2.0):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    q = (torch.randn(Hq, N, d, generator=g) * scale / d ** 0.25).to(torch.bfloat16)
+    k = (torch.randn(Hkv, N, d, generator=g) * scale / d ** 0.25).to(torch.bfloat16)
+    v = torch.randn(Hkv, N, d, generator=g).to(torch.bfloat16)
+    return q, k, v
+
+
+def _sync_ok(ctx):
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+
+
+# ------------------------------------------------------------------ step 1: dense + importance
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("Hq,Hkv,N,d,B", [(4, 2, 512, 64, 64), (4, 1, 640, 128, 128), (2, 2, 384, 128, 64),
+                                          (3, 1, 512, 64, 128), (2, 1, 128, 128, 128)])
+def test_dense_pivot_attn_matches_oracle(binding, kernel, Hq, Hkv, N, d, B):
+    q, k, v = _rand_layer(1, Hq, Hkv, N, d)
+    Q, K, V = par.f64(q), par.f64(k), par.f64(v)
+    ctx = binding.Context(kernel=kernel)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    heads = list(range(Hq))[::-1]            # any order
+    Nb = N // B
+    out = torch.full_like(qd, float("nan"))
+    imp = torch.full((Hq, Nb, Nb), float("nan"), device="cuda")
+    lse = torch.full((Hq, N), float("nan"), device="cuda")
+    ctx.sp_dense_pivot_attn(qd, kd, vd, heads, B, out, importance_out=imp, lse_out=lse)
+    _sync_ok(ctx)
+    for t, h in enumerate(heads):
+        I, O = orc.importance_map(Q, K, V, h, B)
+        par.assert_out_close(par.f64(out[h]), O, f"head {h}")
+        got = imp[t].cpu().numpy().astype(np.float64)
+        assert np.all(np.triu(got, 1) == 0)
+        np.testing.assert_allclose(got, I, rtol=0, atol=par.IMP_ATOL)
+        np.testing.assert_allclose(got.sum(axis=1), 1.0, atol=1e-5)
+        # log-sum-exp of the scaled logits, natural log
+        g = h // (Hq // Hkv)
+        S = (Q[h] @ K[g].T) / np.sqrt(d)
+        S = np.where(np.tril(np.ones((N, N), bool)), S, -np.inf)
+        ref_lse = np.log(np.exp(S - S.max(1, keepdims=True)).sum(1)) + S.max(1)
+        np.testing.assert_allclose(lse[t].cpu().numpy(), ref_lse, atol=2e-3)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_dense_without_importance_and_strided_views(binding, kernel):
+    Hq, Hkv, N, d, B = 4, 2, 256, 128, 128
+    q, k, v = _rand_layer(2, Hq, Hkv, N, d)
+    # K and V interleaved in one buffer, like a fused QKV projection output: [N, 2*Hkv, d]
+    kv = torch.stack([k, v], dim=0).permute(2, 0, 1, 3).contiguous().cuda()   # [N, 2, Hkv, d]
+    kd = kv[:, 0].permute(1, 0, 2)                                             # [Hkv, N, d] strided
+    vd = kv[:, 1].permute(1, 0, 2)
+    ctx = binding.Context(kernel=kernel)
+    out = torch.zeros(Hq, N, d, dtype=torch.bfloat16, device="cuda")
+    ctx.sp_dense_pivot_attn(q.cuda(), kd, vd, [1, 3], B, out)
+    _sync_ok(ctx)
+    ref = orc.dense_causal_attention(par.f64(q), par.f64(k), par.f64(v), B=B, heads=[1, 3])
+    par.assert_out_close(par.f64(out[1]), ref[0])
+    par.assert_out_close(par.f64(out[3]), ref[1])
+    assert torch.all(out[0] == 0) and torch.all(out[2] == 0)                   # unlisted heads untouched
+
+
+# ------------------------------------------------------------------ step 2: importance -> mask
+
+def _mask_case(binding, imp_np, gamma):
+    ctx = binding.Context()
+    n_maps, nb, _ = imp_np.shape
+    imp = torch.from_numpy(imp_np).cuda()
+    mask = torch.full((n_maps, nb, nb), 7, dtype=torch.uint8, device="cuda")
+    counts = torch.full((n_maps, nb), -5, dtype=torch.int32, device="cuda")
+    idx = torch.full((n_maps, nb, nb), -5, dtype=torch.int32, device="cuda")
+    ctx.sp_block_mask_from_importance(imp, gamma, mask, counts, idx)
+    _sync_ok(ctx)
+    g = par.gamma32(gamma)
+    for m in range(n_maps):
+        M, cnt, lists, infos = orc.block_mask_from_importance(imp_np[m].astype(np.float64), g)
+        # the float64 running sum is associated differently on the GPU: a row whose
+        # sum passes within 1e-12 of gamma could differ; none of these inputs has one
+        for i in range(nb):
+            assert min(abs(infos[i]["cum_at_cut"] - g), abs(infos[i]["cum_before_cut"] - g)) > 1e-12 \
+                or infos[i]["cum_at_cut"] == g
+        assert np.array_equal(mask[m].cpu().numpy(), M)
+        assert np.array_equal(counts[m].cpu().numpy(), cnt)
+        got_idx = idx[m].cpu().numpy()
+        for i in range(nb):
+            assert np.array_equal(got_idx[i, :cnt[i]], lists[i])
+            assert np.all(got_idx[i, cnt[i]:] == -1)
+
+
+@pytest.mark.parametrize("nb", [1, 2, 31, 32, 33, 64, 100, 257, 512, 1024])
+def test_block_mask_bit_exact_random(binding, nb):
+    rng = np.random.default_rng(nb)
+    n_maps = 3 if nb <= 257 else 2
+    x = rng.random((n_maps, nb, nb)) ** 6
+    x = np.tril(x)
+    x /= x.sum(axis=2, keepdims=True)
+    x = x.astype(np.float32)
+    x += np.triu(np.full((nb, nb), 0.5, np.float32), 1)      # junk above the diagonal must be ignored
+    for gamma in (0.9, 0.5, 0.999):
+        _mask_case(binding, x, gamma)
+
+
+def test_block_mask_ties_zeros_and_extremes(binding):
+    nb = 40
+    x = np.zeros((4, nb, nb), np.float32)
+    for i in range(nb):
+        x[0, i, :i + 1] = 1.0 / (i + 1)                       # all equal: ties -> lowest indices
+        x[1, i, :i + 1] = 0.0                                  # all zero: never reaches gamma -> everything
+        x[1, i, i // 2] = 0.25
+        x[2, i, :i + 1] = np.float32(2.0) ** -np.arange(1, i + 2)   # exact binary fractions
+        x[3, i, i] = 1.0                                       # one-hot on the diagonal
+    _mask_case(binding, x, 0.75)                               # map 2: 0.5 + 0.25 == 0.75 exactly ('>=')
+    _mask_case(binding, x, 0.9)
+    _mask_case(binding, x, 1.5)                                # unreachable -> every causal tile
+    _mask_case(binding, x, 1e-6)                               # -> the arg-max tile only
+
+
+# ------------------------------------------------------------------ step 3: block-sparse attention
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("Hq,Hkv,N,d,B", [(4, 2, 1024, 64, 64), (4, 1, 1536, 128, 128), (2, 2, 768, 128, 64)])
+def test_block_sparse_attn_matches_oracle(binding, kernel, Hq, Hkv, N, d, B):
+    q, k, v = _rand_layer(3, Hq, Hkv, N, d)
+    Q, K, V = par.f64(q), par.f64(k), par.f64(v)
+    Nb = N // B
+    rng = np.random.default_rng(5)
+    n_lists = 2
+    masks = np.zeros((n_lists, Nb, Nb), np.uint8)
+    for l in range(n_lists):
+        m = np.tril(rng.random((Nb, Nb)) < 0.35).astype(np.uint8)
+        for i in range(Nb):
+            if m[i].sum() == 0:
+                m[i, rng.integers(0, i + 1)] = 1               # never the diagonal by construction
+        masks[l] = m
+    counts = masks.sum(axis=2).astype(np.int32)
+    indices = np.full((n_lists, Nb, Nb), -1, np.int32)
+    for l in range(n_lists):
+        for i in range(Nb):
+            sel = np.nonzero(masks[l, i])[0]
+            indices[l, i, :len(sel)] = sel
+    ctx = binding.Context(kernel=kernel)
+    out = torch.full((Hq, N, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    heads = [2, 0, 3, 1]
+    lists = [1, 0, -1, 1]                                       # head 3 dense
+    ctx.sp_block_sparse_attn(q.cuda(), k.cuda(), v.cuda(), heads, lists, torch.from_numpy(counts).cuda(),
+                             torch.from_numpy(indices).cuda(), B, out)
+    _sync_ok(ctx)
+    for h, l in zip(heads, lists):
+        M = masks[l] if l >= 0 else np.tril(np.ones((Nb, Nb), np.uint8))
+        ref = orc.masked_attention(Q, K, V, h, M, B)
+        par.assert_out_close(par.f64(out[h]), ref, f"head {h}")
+
+
+# ------------------------------------------------------------------ the whole layer
+
+def _run_layer(binding, L, gamma, kernel, row_blocks=None):
+    cfg = L["cfg"]
+    ctx = binding.Context(kernel=kernel)
+    qd, kd, vd = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+    Nb = cfg.seq // cfg.block
+    out = torch.full_like(qd, float("nan"))
+    mask = torch.full((cfg.n_q_heads, Nb, Nb), 9, dtype=torch.uint8, device="cuda")
+    ctx.sp_prefill_attn(qd, kd, vd, L["cluster_map"], L["pivot_heads"], gamma, cfg.block, out, mask_out=mask)
+    _sync_ok(ctx)
+    return out, mask
+
+
+def _check_layer(L, gamma, out, mask, row_blocks=None):
+    cfg = L["cfg"]
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
+    g = par.gamma32(gamma)
+    rows = list(range(Nb)) if row_blocks is None else row_blocks
+    ref = orc.prefill_attn(Q, K, V, L["cluster_map"], L["pivot_heads"], g, B, row_blocks=row_blocks)
+    mask_np = mask.cpu().numpy()
+    bad = exempt = 0
+    src, mask_src = orc.share_masks(L["cluster_map"], L["pivot_heads"])
+    clean_pivot = {}
+    for t, p in enumerate(L["pivot_heads"]):
+        b, e = par.compare_mask_rows(mask_np[p], ref["mask"][p], ref["infos"][t], g, rows)
+        bad += b
+        exempt += e
+        clean_pivot[t] = {i for i in rows if np.array_equal(mask_np[p][i], ref["mask"][p][i])}
+    assert bad == 0, f"{bad} row-blocks differ outside the {par.MASK_BAND} band ({exempt} inside)"
+    worst = (0.0, 0.0)
+    for h in range(cfg.n_q_heads):
+        # members report their pivot's mask, dense heads the causal mask
+        if mask_src[h] >= 0:
+            assert np.array_equal(mask_np[h][rows], mask_np[L["pivot_heads"][mask_src[h]]][rows])
+        else:
+            assert np.array_equal(mask_np[h][rows], np.tril(np.ones((Nb, Nb), np.uint8))[rows])
+        assert np.all(np.triu(mask_np[h], 1) == 0)
+        got = par.f64(out[h])
+        for i in rows:
+            if src[h] >= 0 and i not in clean_pivot[src[h]]:
+                continue                                         # row-block whose mask legitimately flipped
+            sl = slice(i * B, (i + 1) * B)
+            ma, rl = par.out_errors(got[sl], ref["out"][h][sl])
+            worst = (max(worst[0], ma), max(worst[1], rl))
+    assert worst[0] <= par.OUT_MAX_ABS and worst[1] <= par.OUT_REL_L2, worst
+    return worst, exempt
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_prefill_tiny_config_full(binding, kernel):
+    L = synth.make_layer(synth.CONFIGS["tiny"], seed=0)
+    out, mask = _run_layer(binding, L, 0.9, kernel)
+    _check_layer(L, 0.9, out, mask)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("name,seq,gamma", [("llama8b_32k", 4096, 0.9), ("qwen7b_64k", 2048, 0.95),
+                                            ("llama8b_128k", 4096, 0.8)])
+def test_prefill_model_shapes_reduced_seq(binding, kernel, name, seq, gamma):
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=1)
+    out, mask = _run_layer(binding, L, gamma, kernel)
+    _check_layer(L, gamma, out, mask)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_prefill_degenerate_head_sets(binding, kernel):
+    cfg = synth.scaled(synth.CONFIGS["tiny"], 512)
+    L = synth.make_layer(cfg, seed=2)
+    # no pivots at all: every head dense
+    L0 = dict(L, pivot_heads=[])
+    out, mask = _run_layer(binding, L0, 0.9, kernel)
+    _check_layer(L0, 0.9, out, mask)
+    # every head a pivot
+    L1 = dict(L, pivot_heads=list(range(cfg.n_q_heads)))
+    out, mask = _run_layer(binding, L1, 0.9, kernel)
+    _check_layer(L1, 0.9, out, mask)
+    # unclustered heads (-1), a cluster without pivot, two pivots in one cluster (first listed wins)
+    cm = [0, 0, 0, 1, 1, -1, 2, 0]
+    L2 = dict(L, cluster_map=cm, pivot_heads=[2, 0, 3])
+    out, mask = _run_layer(binding, L2, 0.9, kernel)
+    _check_layer(L2, 0.9, out, mask)
+    # gamma beyond reach: every head effectively dense
+    out, mask = _run_layer(binding, L, 1.5, kernel)
+    _check_layer(L, 1.5, out, mask)
+
+
+def test_tc_and_simt_kernels_agree_on_importance(binding):
+    # two different algorithms for the tile mass (one pass + spilled statistics vs two passes)
+    q, k, v = _rand_layer(7, 2, 1, 1024, 128, scale=3.0)
+    res = {}
+    for kernel in KERNELS:
+        ctx = binding.Context(kernel=kernel)
+        out = torch.empty(2, 1024, 128, dtype=torch.bfloat16, device="cuda")
+        imp = torch.empty(2, 8, 8, device="cuda")
+        ctx.sp_dense_pivot_attn(q.cuda(), k.cuda(), v.cuda(), [0, 1], 128, out, importance_out=imp)
+        _sync_ok(ctx)
+        res[kernel] = imp.cpu().numpy()
+    np.testing.assert_allclose(res["tc"], res["simt"], rtol=0, atol=par.IMP_ATOL)
+
+
+# ------------------------------------------------------------------ argument checking (host side)
+
+def test_invalid_arguments_are_rejected(binding):
+    ctx = binding.Context()
+    q = torch.zeros(4, 256, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(2, 256, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(q)
+
+    def code(fn):
+        with pytest.raises(binding.SpError) as e:
+            fn()
+        return e.value.code
+
+    assert code(lambda: ctx.sp_dense_pivot_attn(q, k, k, [0], 32, out)) == binding.SP_ERR_UNSUPPORTED      # block
+    assert code(lambda: ctx.sp_dense_pivot_attn(q, k, k, [4], 128, out)) == binding.SP_ERR_INVALID_ARG     # head range
+    assert code(lambda: ctx.sp_dense_pivot_attn(q[:, :200], k[:, :200], k[:, :200], [0], 128, out[:, :200])) \
+        == binding.SP_ERR_UNSUPPORTED                                                                      # ragged seq
+    k3 = torch.zeros(3, 256, 128, dtype=torch.bfloat16, device="cuda")
+    assert code(lambda: ctx.sp_dense_pivot_attn(q, k3, k3, [0], 128, out)) == binding.SP_ERR_UNSUPPORTED   # 4 % 3
+    q96 = torch.zeros(4, 256, 96, dtype=torch.bfloat16, device="cuda")
+    k96 = torch.zeros(2, 256, 96, dtype=torch.bfloat16, device="cuda")
+    assert code(lambda: ctx.sp_dense_pivot_attn(q96, k96, k96, [0], 128, torch.zeros_like(q96))) == binding.SP_ERR_UNSUPPORTED
+    assert code(lambda: ctx.sp_dense_pivot_attn(q, k, k[:, :128], [0], 128, out)) == binding.SP_ERR_INVALID_ARG
+    assert code(lambda: ctx.sp_prefill_attn(q, k, k, [0, 0, 1, 1], [0, 0], 0.9, 128, out)) == binding.SP_ERR_INVALID_ARG  # dup
+    assert code(lambda: ctx.sp_prefill_attn(q, k, k, [0, 0, 1, 1], [0], 0.0, 128, out)) == binding.SP_ERR_INVALID_ARG
+    imp = torch.zeros(1, 8, 8, device="cuda")
+    cnt = torch.zeros(1, 8, dtype=torch.int32, device="cuda")
+    idx = torch.zeros(1, 8, 8, dtype=torch.int32, device="cuda")
+    assert code(lambda: ctx.sp_block_mask_from_importance(imp, -1.0, None, cnt, idx)) == binding.SP_ERR_INVALID_ARG
+    assert code(lambda: ctx.sp_block_sparse_attn(q, k, k, [0], [3], cnt, idx, 128, out)) == binding.SP_ERR_INVALID_ARG
+    # nothing was launched and the context is still fine
+    ctx.sp_dense_pivot_attn(q, k, k, [], 128, out)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
