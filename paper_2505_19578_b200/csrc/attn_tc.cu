@@ -1,4 +1,493 @@
+// Tensor-core attention kernel for sm_100a: dense (pivot) and block-sparse
+// (member) causal attention in one template.
+//
+//   Section 5.1:  O = softmax(Q K^T / sqrt(d) - c (1 - M)) V,  c -> infinity,
+//   causal.  A pivot walks every causal key-block and also emits the softmax
+//   probability mass of each (query-block, key-block) tile; a member walks the
+//   compacted list of key-blocks its cluster's pivot selected.
+//
+// One CTA owns one (head, query row-block).  Warp roles:
+//   warps 0-3  softmax: thread t owns query row t = TMEM lane t.  Reads S from
+//              TMEM, keeps the running max / sum, writes P (bf16) back into the
+//              columns S occupied, rescales the O accumulator when the running
+//              max moved, and runs the epilogue.
+//   warp 4     producer: TMA loads of Q (once) and of one K and one V tile per
+//              step into 128-byte-swizzled shared memory.
+//   warp 5     MMA issuer: S = Q K^T (both operands from shared memory) and
+//              O += P V (P from TMEM, V from shared memory, N-major), bf16 in,
+//              fp32 accumulate in TMEM.  Owns the TMEM allocation.
+// K and V have one shared-memory slot each: the K slot is free as soon as
+// Q K^T has been read (long before the next step needs it), the V slot as soon
+// as P V has.  Two CTAs share an SM, so one CTA's softmax overlaps the other's
+// MMAs.
+//
+// Block importance in one pass: for each visited tile the softmax thread spills
+// one float per row, stat = m + log2(sum_c 2^(s_c - m)) with m the row's running
+// reference max at that step.  After the last tile the row's final log-sum-exp
+// L is known and the tile mass is (1/B) sum_rows 2^(stat - L).
+//
+// Every wait on an mbarrier is bounded: when it runs out the CTA raises an abort
+// flag, records SP_ERR_TIMEOUT in the status word, and all roles fall through
+// to the common teardown (TMEM is freed, the kernel returns).
+#include <cuda.h>
+#include <math_constants.h>
+
 #include "common.cuh"
+
 namespace sp {
-cudaError_t launch_attn_tc(const AttnArgs&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 1000000000ll;  // ~0.5 s at 2 GHz; a step takes microseconds
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+struct Abort {
+  volatile int* flag;  // shared memory
+  int* status;         // global int[2]
+};
+
+// Bounded wait.  Returns false if the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*ab.flag) return false;
+      if (*reinterpret_cast<volatile int*>(ab.status) != 0) {   // another CTA already gave up
+        *ab.flag = 1;
+        return false;
+      }
+      if (clock64() - t0 > kWaitCycles) break;
+    }
+  }
+  *ab.flag = 1;
+  if (atomicCAS(ab.status, 0, (int)SP_ERR_TIMEOUT) == 0) ab.status[1] = where;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane -> registers (waits for the data).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+// registers -> 32 consecutive 32-bit columns of this thread's TMEM lane (does not wait).
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M x N, operand majors (0 = K-major, 1 = MN-major).
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ shared-memory plan
+
+template <int D, int BLK>
+struct Plan {
+  static constexpr int NBOX = D / 64;          // 64-column (128-byte) boxes per row
+  static constexpr int QBOX = 128 * 128;       // bytes of one Q box: the MMA reads 128 rows
+  static constexpr int KBOX = BLK * 128;       // bytes of one K / V box
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = Q_OFF + NBOX * QBOX;
+  static constexpr int V_OFF = K_OFF + NBOX * KBOX;
+  static constexpr int MISC_OFF = V_OFF + NBOX * KBOX;
+  static constexpr int MISC_BYTES = 1024;
+  static constexpr int TOTAL = MISC_OFF + MISC_BYTES + 1024;   // + slack for 1024-byte alignment
+  static constexpr int Q_TX = NBOX * BLK * 128;                 // bytes the Q loads deliver
+  static constexpr int KV_TX = NBOX * KBOX;
+  static constexpr int TMEM_COLS = (BLK + D) <= 128 ? 128 : 256;
+  static constexpr int S_COL = 0;              // S (fp32, BLK columns); P (bf16 pairs) reuses its first BLK/2
+  static constexpr int O_COL = BLK;            // O accumulator (fp32, D columns)
+};
+
+// barrier slots inside the MISC area
+enum { BAR_Q_FULL = 0, BAR_K_FULL, BAR_V_FULL, BAR_QK_DONE, BAR_P_FULL, BAR_PV_DONE, BAR_COUNT };
+
+template <int D, int BLK>
+__global__ void __launch_bounds__(kThreads, 2)
+attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v) {
+  using P = Plan<D, BLK>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sQ = smem_u32(smem + P::Q_OFF), sK = smem_u32(smem + P::K_OFF), sV = smem_u32(smem + P::V_OFF);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + P::MISC_OFF);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + P::MISC_OFF + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + P::MISC_OFF + 72);
+  float* lse_smem = reinterpret_cast<float*>(smem + P::MISC_OFF + 128);   // 128 floats
+  auto bar = [&](int which) { return smem_u32(bars + which); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i = a.Nb - 1 - (int)blockIdx.x;      // long row-blocks first
+  const int slot = blockIdx.y;
+  const int h = a.heads.v[slot];
+  const int g = h / a.group;
+  const int list = a.lists.v[slot];
+  int cnt = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
+  cnt = cnt < 0 ? 0 : (cnt > i + 1 ? i + 1 : cnt);
+  const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
+  if (poisoned) cnt = 0;
+  const int32_t* idx = list >= 0 ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;
+  const bool emit = a.importance != nullptr && list < 0;
+  const Abort ab{abort_flag, a.status};
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(BAR_Q_FULL), 1);
+    mbar_init(bar(BAR_K_FULL), 1);
+    mbar_init(bar(BAR_V_FULL), 1);
+    mbar_init(bar(BAR_QK_DONE), 1);
+    mbar_init(bar(BAR_P_FULL), 128);
+    mbar_init(bar(BAR_PV_DONE), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (BLK < 128) {
+    // rows BLK..127 of the Q operand are never loaded: make them zeros
+    for (int b = 0; b < P::NBOX; ++b) {
+      uint4* z = reinterpret_cast<uint4*>(smem + P::Q_OFF + b * P::QBOX + BLK * 128);
+      for (int x = threadIdx.x; x < (128 - BLK) * 128 / 16; x += kThreads) z[x] = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(tmem_slot), P::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0 && cnt > 0) {
+      mbar_expect_tx(bar(BAR_Q_FULL), P::Q_TX);
+      for (int b = 0; b < P::NBOX; ++b) tma_load_3d(sQ + b * P::QBOX, &tm_q, bar(BAR_Q_FULL), b * 64, i * BLK, h);
+      int issued_k = 0, issued_v = 0;
+      bool ok = true;
+      for (int t = 0; t < cnt && ok; ++t) {
+        const int j = idx ? idx[t] : t;
+        if (t > 0) ok = mbar_wait(bar(BAR_QK_DONE), (t - 1) & 1, ab, 10);
+        if (!ok) break;
+        mbar_expect_tx(bar(BAR_K_FULL), P::KV_TX);
+        for (int b = 0; b < P::NBOX; ++b) tma_load_3d(sK + b * P::KBOX, &tm_k, bar(BAR_K_FULL), b * 64, j * BLK, g);
+        ++issued_k;
+        if (t > 0) ok = mbar_wait(bar(BAR_PV_DONE), (t - 1) & 1, ab, 11);
+        if (!ok) break;
+        mbar_expect_tx(bar(BAR_V_FULL), P::KV_TX);
+        for (int b = 0; b < P::NBOX; ++b) tma_load_3d(sV + b * P::KBOX, &tm_v, bar(BAR_V_FULL), b * 64, j * BLK, g);
+        ++issued_v;
+      }
+      if (*abort_flag) {
+        // let the copies already in flight land before the CTA gives its shared memory back
+        const long long t0 = clock64();
+        while (clock64() - t0 < kWaitCycles / 8) {
+          bool done = mbar_try_wait(bar(BAR_Q_FULL), 0);
+          if (issued_k) done = done && mbar_try_wait(bar(BAR_K_FULL), (issued_k - 1) & 1);
+          if (issued_v) done = done && mbar_try_wait(bar(BAR_V_FULL), (issued_v - 1) & 1);
+          if (done) break;
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc_qk = instr_desc(128, BLK, 0, 0);
+    constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
+    bool ok = cnt > 0 ? mbar_wait(bar(BAR_Q_FULL), 0, ab, 20) : false;
+    for (int t = 0; t < cnt && ok; ++t) {
+      ok = mbar_wait(bar(BAR_K_FULL), t & 1, ab, 21);
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * P::QBOX + (kk & 3) * 32;
+          const uint32_t koff = (kk >> 2) * P::KBOX + (kk & 3) * 32;
+          mma_ss(tmem + P::S_COL, smem_desc(sQ + off, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, kk > 0);
+        }
+        mma_commit(bar(BAR_QK_DONE));
+      }
+      __syncwarp();
+      ok = mbar_wait(bar(BAR_P_FULL), t & 1, ab, 22) && mbar_wait(bar(BAR_V_FULL), t & 1, ab, 23);
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+#pragma unroll
+        for (int kk = 0; kk < BLK / 16; ++kk) {
+          // V tile: rows = keys (the MMA's K), 128-byte rows of 64 head-dim columns per box (N-major)
+          mma_ts(tmem + P::O_COL, tmem + P::S_COL + kk * 8, smem_desc(sV + kk * 16 * 128, P::KBOX, 1024), idesc_pv,
+                 (t > 0 || kk > 0) ? 1u : 0u);
+        }
+        mma_commit(bar(BAR_PV_DONE));
+      }
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue
+    const int row = threadIdx.x;                       // TMEM lane == query row inside the tile
+    const bool row_valid = row < BLK;
+    const int r = i * BLK + (row_valid ? row : 0);
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    const float scale = a.scale_log2;
+    float* stats = emit ? a.tile_stats + ((size_t)slot * ((size_t)a.Nb * (a.Nb + 1) / 2) + (size_t)i * (i + 1) / 2) * BLK
+                        : nullptr;
+    float m_ref = -CUDART_INF_F, l = 0.f;
+    bool ok = cnt > 0;
+    for (int t = 0; t < cnt && ok; ++t) {
+      const int j = idx ? idx[t] : t;
+      ok = mbar_wait(bar(BAR_QK_DONE), t & 1, ab, 30);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s[BLK];
+#pragma unroll
+      for (int c = 0; c < BLK / 32; ++c) tmem_ld32(tl + P::S_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      float mx = -CUDART_INF_F;
+      if (j == i) {
+#pragma unroll
+        for (int c = 0; c < BLK; ++c) {
+          float x = c > row ? -CUDART_INF_F : __uint_as_float(s[c]);
+          s[c] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < BLK; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+      }
+      mx *= scale;
+      // the reference max only moves when the row max has grown by more than 2^8
+      const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+      const float alpha = ex2_approx(m_ref - m_new);
+      float sum = 0.f;
+      uint32_t p[BLK / 2];
+#pragma unroll
+      for (int c = 0; c < BLK; c += 2) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), scale, -m_new));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), scale, -m_new));
+        sum += p0 + p1;
+        p[c / 2] = pack_bf16(p0, p1);
+      }
+      l = l * alpha + sum;
+      if (emit && row_valid) stats[(size_t)t * BLK + row] = m_new + log2f(sum);
+      if (t > 0 && __any_sync(0xffffffffu, m_new != m_ref)) {
+        // O of the previous steps is relative to the old reference: bring it to the new one
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tl + P::O_COL + c * 32, o);
+#pragma unroll
+          for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
+          tmem_st32(tl + P::O_COL + c * 32, o);
+        }
+      }
+      m_ref = m_new;
+#pragma unroll
+      for (int c = 0; c < BLK / 64; ++c) tmem_st32(tl + P::S_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p[c * 32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_P_FULL));
+    }
+    if (ok) ok = mbar_wait(bar(BAR_PV_DONE), (cnt - 1) & 1, ab, 31);
+    if (ok) {
+      tc_fence_after();
+      const float inv_l = 1.f / l;
+      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tl + P::O_COL + c * 32, o);
+        if (row_valid) {
+          uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            uint4 u;
+            u.x = pack_bf16(__uint_as_float(o[8 * x + 0]) * inv_l, __uint_as_float(o[8 * x + 1]) * inv_l);
+            u.y = pack_bf16(__uint_as_float(o[8 * x + 2]) * inv_l, __uint_as_float(o[8 * x + 3]) * inv_l);
+            u.z = pack_bf16(__uint_as_float(o[8 * x + 4]) * inv_l, __uint_as_float(o[8 * x + 5]) * inv_l);
+            u.w = pack_bf16(__uint_as_float(o[8 * x + 6]) * inv_l, __uint_as_float(o[8 * x + 7]) * inv_l);
+            dst[x] = u;
+          }
+        }
+      }
+      const float lse2 = m_ref + log2f(l);
+      if (a.lse && row_valid) a.lse[(size_t)slot * a.N + r] = lse2 * 0.6931471805599453f;
+      if (emit) {
+        lse_smem[row] = lse2;
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // the four softmax warps: statistics and lse visible
+        float* imp_row = a.importance + ((size_t)slot * a.Nb + i) * a.Nb;
+        for (int t = warp; t < cnt; t += 4) {
+          float acc = 0.f;
+          for (int rr = lane; rr < BLK; rr += 32) acc += exp2f(stats[(size_t)t * BLK + rr] - lse_smem[rr]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          if (lane == 0) imp_row[t] = acc * (1.f / BLK);
+        }
+        for (int jz = i + 1 + (int)threadIdx.x; jz < a.Nb; jz += 128) imp_row[jz] = 0.f;
+      }
+    } else if (cnt == 0 && row_valid && !poisoned) {
+      // an empty list is outside the contract; leave defined output (zeros) rather than garbage
+      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+      for (int x = 0; x < D / 8; ++x) reinterpret_cast<uint4*>(orow)[x] = make_uint4(0, 0, 0, 0);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, P::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [heads, seq, dim] bf16 view -> 3-D tensor map with a (64 columns x box_rows x 1) box, 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* base, int64_t sh, int64_t sn, int H, int N, int d, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if (H == 1 || sh == 0) sh = (int64_t)N * sn;
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H};
+  cuuint64_t strides[2] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int BLK>
+cudaError_t launch(const AttnArgs& a, cudaStream_t s) {
+  using P = Plan<D, BLK>;
+  CUtensorMap tq, tk, tv;
+  if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
+      !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK) ||
+      !make_map(&tv, a.v, a.v_sh, a.v_sn, a.n_kv_heads, a.N, D, BLK))
+    return cudaErrorInvalidValue;
+  // at most two CTAs per SM (their TMEM allocations must both fit in 512 columns)
+  constexpr int smem = P::TOTAL > 100 * 1024 ? P::TOTAL : 100 * 1024;
+  cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, BLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  attn_tc_kernel<D, BLK><<<dim3(a.Nb, a.n_heads), kThreads, smem, s>>>(a, tq, tk, tv);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s) {
+  if (a.d == 128 && a.B == 128) return launch<128, 128>(a, s);
+  if (a.d == 128 && a.B == 64) return launch<128, 64>(a, s);
+  if (a.d == 64 && a.B == 128) return launch<64, 128>(a, s);
+  if (a.d == 64 && a.B == 64) return launch<64, 64>(a, s);
+  return cudaErrorInvalidValue;
+}
+
 }  // namespace sp

@@ -163,8 +163,8 @@ def test_block_sparse_attn_matches_oracle(binding, kernel, Hq, Hkv, N, d, B):
             indices[l, i, :len(sel)] = sel
     ctx = binding.Context(kernel=kernel)
     out = torch.full((Hq, N, d), float("nan"), dtype=torch.bfloat16, device="cuda")
-    heads = [2, 0, 3, 1]
-    lists = [1, 0, -1, 1]                                       # head 3 dense
+    heads = [2, 0, 3, 1] if Hq == 4 else [1, 0]
+    lists = [1, 0, -1, 1] if Hq == 4 else [-1, 1]              # one head dense (list -1)
     ctx.sp_block_sparse_attn(q.cuda(), k.cuda(), v.cuda(), heads, lists, torch.from_numpy(counts).cuda(),
                              torch.from_numpy(indices).cuda(), B, out)
     _sync_ok(ctx)
