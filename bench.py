@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the SharePrefill prefill-attention layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload llama8b_128k] [--gamma 0.9] [--seed 0]
+
+A "step" is one whole pass of the hot path (pivot dense attention + block
+importance, importance -> mask, block-sparse attention of the member heads)
+over one synthetic layer, i.e. one `sp_prefill_attn` call.  Prints ONE JSON
+line.  `value` is effective (as-if-dense) TFLOP/s:
+Hq * 4 d * N (N + 1) / 2 flops per layer divided by the time of a layer.
+
+With N > 1 (torchrun, one process per GPU) every rank runs its own layer
+(independent problems: different seeds, as the layers of a model are), no
+data-path collective; the time is the max over ranks and `value` the sum of the
+layers done divided by it ("weak" scaling).
+
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same
+workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2505_19578_b200 import synth  # noqa: E402
+
+METRIC = "effective_tflops_prefill_attention_layer"
+UNIT = "TFLOP/s"
+
+
+# ----------------------------------------------------------------------------- helpers (host logic, CPU-testable)
+
+def dense_flops(cfg) -> float:
+    """As-if-dense causal attention flops of one layer: Hq * 4 d * N (N+1) / 2."""
+    return cfg.n_q_heads * 4.0 * cfg.head_dim * cfg.seq * (cfg.seq + 1) / 2.0
+
+
+def tile_flops(cfg) -> float:
+    """QK^T + PV of one full (block x block) tile."""
+    return 4.0 * cfg.block * cfg.block * cfg.head_dim
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each rank works on its own layer (independent problem)."""
+    return base_seed + 1000 * rank
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate(ms_local: float, layers_local: float, world: int, device=None):
+    """Max time over ranks, total layers over ranks."""
+    if world == 1:
+        return ms_local, layers_local
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([layers_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item())
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "hbm_gbs": d["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power),
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_sample_time(L, gamma, row_blocks):
+    """Times the float64 oracle (as it stands) on the given row-blocks of every head.
+    Returns (seconds, as-if-dense flops covered, threads used)."""
+    import numpy as np
+    from oracle import shareprefill_oracle as orc
+    cfg = L["cfg"]
+    Q = L["q"].float().cpu().numpy().astype(np.float64)
+    K = L["k"].float().cpu().numpy().astype(np.float64)
+    V = L["v"].float().cpu().numpy().astype(np.float64)
+    g = float(np.float32(gamma))
+    t0 = time.perf_counter()
+    orc.prefill_attn(Q, K, V, L["cluster_map"], L["pivot_heads"], g, cfg.block, row_blocks=row_blocks)
+    dt = time.perf_counter() - t0
+    B, d = cfg.block, cfg.head_dim
+    flops = sum(cfg.n_q_heads * 4.0 * d * B * (i * B + (B + 1) / 2.0) for i in row_blocks)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return dt, flops, threads
+
+
+def workload_cfg(args):
+    cfg = synth.CONFIGS[args.workload]
+    return synth.scaled(cfg, args.seq) if args.seq else cfg
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    cfg = workload_cfg(args)
+    L = synth.make_layer(cfg, seed=rank_seed(args.seed, 0), device="cpu")
+    Nb = cfg.seq // cfg.block
+    rbs = [Nb // 2]
+    times, flops, threads = [], 0.0, 1
+    for s in range(args.warmup + args.steps):
+        dt, flops, threads = oracle_sample_time(L, args.gamma, rbs)
+        if s >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = flops / (ms * 1e-3) / 1e12
+    sample = f"row-block {rbs[0]} of {Nb} for all {cfg.n_q_heads} heads per step (float64 numpy oracle)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "block": cfg.block, "gamma": args.gamma, "seed": args.seed},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+def run_ours(args):
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2505_19578_b200 import binding, build
+    build.build()
+
+    cfg = workload_cfg(args)
+    gamma = args.gamma
+    L = synth.make_layer(cfg, seed=rank_seed(args.seed, rank), device=str(dev))
+    q, k, v = L["q"], L["k"], L["v"]
+    cm, piv = L["cluster_map"], L["pivot_heads"]
+    Nb, B = cfg.seq // cfg.block, cfg.block
+    ctx = binding.Context(device=local_rank)
+    ctx.reserve(binding.workspace_bytes(cfg.seq, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, B, len(piv)))
+    out = torch.empty_like(q)
+    mask = torch.empty(cfg.n_q_heads, Nb, Nb, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, B, out, mask_out=mask, stream=stream)
+
+    # ---- warm-up, then the timed region: K whole-layer steps, inputs resident in HBM
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_local = e0.elapsed_time(e1) / args.steps
+    launches = ctx.launch_count() - launches0
+    assert ctx.status() == (0, 0), "device-side wait timed out"
+
+    # ---- per-kernel split: the same step issued as its three public calls with events between
+    members = [h for h in range(cfg.n_q_heads) if h not in piv]
+    first_pivot_of = {}
+    for t, p in enumerate(piv):
+        first_pivot_of.setdefault(cm[p], t)
+    lists = [first_pivot_of.get(cm[h], -1) if cm[h] >= 0 else -1 for h in members]
+    imp = torch.empty(len(piv), Nb, Nb, device=dev)
+    pm = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device=dev)
+    counts = torch.empty(len(piv), Nb, dtype=torch.int32, device=dev)
+    indices = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device=dev)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+
+    def split_step(e):
+        e[0].record(stream)
+        ctx.sp_dense_pivot_attn(q, k, v, piv, B, out, importance_out=imp, stream=stream)
+        e[1].record(stream)
+        ctx.sp_block_mask_from_importance(imp, gamma, pm, counts, indices, stream=stream)
+        e[2].record(stream)
+        ctx.sp_block_sparse_attn(q, k, v, members, lists, counts, indices, B, out, stream=stream)
+        e[3].record(stream)
+
+    scratch = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    split_step(scratch)
+    torch.cuda.synchronize()
+    for e in ev:
+        split_step(e)
+    torch.cuda.synchronize()
+    k1 = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    k2 = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    k3 = sum(e[2].elapsed_time(e[3]) for e in ev) / args.steps
+    cnt_host = counts.cpu().numpy()
+    tiles_causal = Nb * (Nb + 1) // 2
+    pivot_tiles = len(piv) * tiles_causal
+    member_tiles = int(sum(int(cnt_host[l].sum()) if l >= 0 else tiles_causal for l in lists))
+    density = {int(p): float(cnt_host[t].sum()) / tiles_causal for t, p in enumerate(piv)}
+
+    # ---- the build's own dense baseline: every head dense, no importance (one warm run, two timed)
+    all_heads = list(range(cfg.n_q_heads))
+    dense_ms = None
+    if rank == 0 and not args.no_dense:
+        ctx.sp_dense_pivot_attn(q, k, v, all_heads, B, out, stream=stream)
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(2):
+            ctx.sp_dense_pivot_attn(q, k, v, all_heads, B, out, stream=stream)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dense_ms = d0.elapsed_time(d1) / 2
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the C ABI with host buffers: H2D of q,k,v, the layer, D2H of the output
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True)
+        dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True)
+        ctx.sp_prefill_attn(dq, dk, dv, cm, piv, gamma, B, out, mask_out=None, stream=stream)
+        hout.copy_(out, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record(stream)
+    barrier()
+    e2e_ms_local = f0.elapsed_time(f1) / e2e_steps
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+    d2h = hout.numel() * hout.element_size()
+
+    ms, layers = aggregate(ms_local, 1.0, world, dev)
+    e2e_ms, _ = aggregate(e2e_ms_local, 1.0, world, dev)
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    F = dense_flops(cfg)
+    Ft = tile_flops(cfg)
+    value = layers * F / (ms * 1e-3) / 1e12
+    k1_tf = pivot_tiles * Ft / (k1 * 1e-3) / 1e12
+    k3_tf = member_tiles * Ft / (k3 * 1e-3) / 1e12 if k3 > 0 else 0.0
+    # dominant kernel by time
+    dom = ("pivot_dense_attn", k1, k1_tf) if k1 >= k3 else ("block_sparse_attn", k3, k3_tf)
+    roofline = {
+        "kernel": f"attn_tc_kernel<{cfg.head_dim},{cfg.block}> ({dom[0]})", "bound": "tensor", "achieved": dom[2],
+        "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": dom[2] / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
+        "peak_kind": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
+        "frac_of_burst_peak": dom[2] / peaks["bf16_tflops"], "traffic": None,
+        "ms_per_launch": dom[1], "flops_per_launch": (pivot_tiles if dom[0].startswith("pivot") else member_tiles) * Ft,
+        "timing": "CUDA events around each of the three public calls, same inputs, same number of steps",
+    }
+    mask_bytes = len(piv) * Nb * Nb * (4 + 1 + 4) + len(piv) * Nb * 4
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "block": cfg.block, "gamma": gamma, "n_pivots": len(piv),
+                   "seed": args.seed, "l2": "inputs (2.5 GiB at 128K) exceed the 126 MB L2; no flush between steps",
+                   "units_per_rank": "one layer per rank, independent seeds"},
+        "ms_per_layer": ms,
+        "kernels_ms": {"pivot_dense_attn": k1, "block_mask": k2, "block_sparse_attn": k3},
+        "visited_tiles": {"pivot": pivot_tiles, "members": member_tiles, "causal_per_head": tiles_causal},
+        "mask_density_per_pivot": density,
+        "visited_tflops": {"pivot_dense_attn": k1_tf, "block_sparse_attn": k3_tf,
+                           "layer": (pivot_tiles + member_tiles) * Ft / (ms * 1e-3) / 1e12},
+        "frac_of_bf16_peak": {"pivot_dense_attn": k1_tf / peaks["bf16_tflops"],
+                              "block_sparse_attn": k3_tf / peaks["bf16_tflops"], "peak": peaks["bf16_tflops"],
+                              "peak_source": peaks["source"]},
+        "block_mask_gbs": mask_bytes / (k2 * 1e-3) / 1e9 if k2 > 0 else None,
+        "dense_baseline_ms": dense_ms,
+        "dense_baseline_tflops": F / (dense_ms * 1e-3) / 1e12 if dense_ms else None,
+        "speedup_vs_dense": dense_ms / ms if dense_ms else None,
+        "roofline": roofline,
+        "e2e": {"value": layers * F / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        Lh = {"q": hq, "k": hk, "v": hv, "cluster_map": cm, "pivot_heads": piv, "cfg": cfg}
+        rbs = sorted({0, Nb // 4, Nb // 2, Nb - 1})
+        dt, fl, threads = oracle_sample_time(Lh, gamma, rbs)
+        result["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                  "seconds": dt,
+                                  "sample": f"row-blocks {rbs} of {Nb} for all {cfg.n_q_heads} heads "
+                                            f"(float64 numpy oracle, whole method)"}
+    print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--gamma", type=float, default=0.9)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
