@@ -58,7 +58,8 @@ enum {
   SP_ERR_UNSUPPORTED = -2, /* a size outside the supported set listed above            */
   SP_ERR_WORKSPACE = -3,   /* workspace allocation failed                              */
   SP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                      */
-  SP_ERR_TIMEOUT = -5      /* a bounded device-side wait ran out (see sp_get_status)   */
+  SP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (see sp_get_status)   */
+  SP_ERR_SCRATCH_LIMIT = -6 /* sp_dense_pivot_attn_fixed_scratch: problem too large for the fixed array */
 };
 
 /* bf16 tensor view: device pointer, sizes and strides in ELEMENTS. */
@@ -112,6 +113,45 @@ const char* sp_strerror(int code);
 int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
                         const int32_t* heads, int n_heads, int block, sp_tensor* out,
                         float* importance_out, float* lse_out, void* stream);
+
+/*
+ * Step 1 again, for callers that must not allocate device memory.
+ *   (The paper has no counterpart: this is a deployment variant of the call above.)
+ *
+ *   Some hosts cannot call cudaMalloc at the moment they need attention: an
+ *   inference-engine plugin whose enqueue hook is forbidden to allocate, a server
+ *   whose memory pool already owns the whole device so that a raw allocation
+ *   fails, a latency-critical loop that cannot afford the device-wide
+ *   synchronisation an allocation implies.  sp_dense_pivot_attn needs a context
+ *   (allocated) and a workspace (allocated, grown on demand) for the per-tile
+ *   softmax statistics behind the importance map.  This variant needs neither:
+ *   it takes no context and keeps those statistics in an array that is part of
+ *   the library image, SP_FIXED_SCRATCH_BYTES (64 MiB) on every GPU that loads the
+ *   library, held until the process exits.  It calls no cudaMalloc / cudaFree and
+ *   no allocating library routine.
+ *
+ *   Same arguments and results as sp_dense_pivot_attn, plus `device`, the CUDA
+ *   device the tensors live on.  Limits and rules:
+ *   - with importance_out != NULL the launch needs
+ *     n_heads * Nb * (Nb + 1) / 2 * block * 4 bytes of statistics; beyond 64 MiB the
+ *     call returns SP_ERR_SCRATCH_LIMIT and launches nothing (e.g. seq 16384, block
+ *     128: 15 heads per call; seq 32768: 3 heads).  Without importance no scratch
+ *     is used and there is no limit.
+ *   - the first call on a device looks up the array's device address (a host-side
+ *     query, done with that device current).  Make that first call outside any
+ *     stream capture.
+ *   - all calls on a device share the one array and one status word.  The array
+ *     keeps whatever the last call left in it; nothing in it needs to start at
+ *     zero, and the status word is cleared on the stream before every launch.
+ *     Two calls whose kernels may run at the same time on the same device
+ *     (different streams, or different host threads) race on it: serialise them.
+ *   - a device-side wait that runs out makes the kernel stop early, as in the
+ *     context version, but this variant has no call to read the status word back.
+ */
+#define SP_FIXED_SCRATCH_BYTES (64ull << 20)
+int sp_dense_pivot_attn_fixed_scratch(int device, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                                      const int32_t* heads, int n_heads, int block, sp_tensor* out,
+                                      float* importance_out, float* lse_out, void* stream);
 
 /*
  * Step 2 - importance map -> block mask and compacted key-block lists.

@@ -22,11 +22,13 @@ SP_ERR_UNSUPPORTED = -2
 SP_ERR_WORKSPACE = -3
 SP_ERR_CUDA = -4
 SP_ERR_TIMEOUT = -5
+SP_ERR_SCRATCH_LIMIT = -6
+FIXED_SCRATCH_BYTES = 64 << 20
 
 EXPORTS = (
     "sp_ctx_create", "sp_ctx_destroy", "sp_workspace_bytes", "sp_ctx_reserve", "sp_get_status",
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
-    "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count",
+    "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
 )
 
 
@@ -64,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.sp_strerror.argtypes = [I]
     lib.sp_strerror.restype = ctypes.c_char_p
     lib.sp_dense_pivot_attn.argtypes = [P, T, T, T, IP, I, I, T, P, P, P]
+    lib.sp_dense_pivot_attn_fixed_scratch.argtypes = [I, T, T, T, IP, I, I, T, P, P, P]
     lib.sp_block_mask_from_importance.argtypes = [P, P, I, I, F, P, P, P, P]
     lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
     lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
@@ -177,6 +180,26 @@ class Context:
         _check(self._lib.sp_prefill_attn(self._h, _view(q), _view(k), _view(v), _i32(cluster_map), _i32(pivot_heads),
                                          len(pivot_heads), gamma, block, _view(out), _ptr(mask_out), _stream(stream)),
                "sp_prefill_attn")
+
+
+def sp_dense_pivot_attn_fixed_scratch(q, k, v, heads, block, out, importance_out=None, lse_out=None, stream=None,
+                                      device=None):
+    """Dense pivot attention + block importance without any device allocation.
+
+    For hosts that may not allocate when they need attention (an engine plugin's
+    enqueue hook, a server whose pool owns the whole device, a latency-critical
+    loop): no context, and the per-tile statistics live in a 64 MiB array inside
+    the library image instead of a workspace.  Raises SpError(SP_ERR_SCRATCH_LIMIT)
+    when n_heads * Nb * (Nb + 1) / 2 * block * 4 bytes exceed that array.  Calls on
+    one device share the array: do not let two of them overlap on the GPU.  The
+    first call on a device resolves the array's address; make it outside stream
+    capture.
+    """
+    heads = list(heads)
+    dev = q.device.index if device is None else int(device)
+    _check(load().sp_dense_pivot_attn_fixed_scratch(dev, _view(q), _view(k), _view(v), _i32(heads), len(heads), block,
+                                                    _view(out), _ptr(importance_out), _ptr(lse_out), _stream(stream)),
+           "sp_dense_pivot_attn_fixed_scratch")
 
 
 def workspace_bytes(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots) -> int:

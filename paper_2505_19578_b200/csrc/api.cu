@@ -163,6 +163,7 @@ const char* sp_strerror(int code) {
     case SP_ERR_WORKSPACE: return "workspace allocation failed";
     case SP_ERR_CUDA: return "CUDA call failed";
     case SP_ERR_TIMEOUT: return "device-side wait timed out";
+    case SP_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's fixed scratch array holds";
     default: return "unknown error code";
   }
 }
@@ -255,6 +256,31 @@ int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, con
     a.tile_stats = static_cast<float*>(ctx->ws);
   }
   return launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+int sp_dense_pivot_attn_fixed_scratch(int device, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                                      const int32_t* heads, int n_heads, int block, sp_tensor* out,
+                                      float* importance_out, float* lse_out, void* stream) {
+  if (!heads || n_heads < 0) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  for (int t = 0; t < n_heads; ++t)
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+  if (importance_out && (size_t)n_heads * tile_stats_bytes_per_head(p.Nb, p.B) > kFixedScratchBytes)
+    return SP_ERR_SCRATCH_LIMIT;
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(device);
+  if (!g.ok) return SP_ERR_CUDA;
+  sp_ctx no_ctx;                       // only so that base_args has somewhere to read a status pointer from
+  AttnArgs a = base_args(&no_ctx, p, q, k, v, out);
+  a.n_heads = n_heads;
+  for (int t = 0; t < n_heads; ++t) { a.heads.v[t] = heads[t]; a.lists.v[t] = -1; }
+  a.importance = importance_out;
+  a.lse = lse_out;
+  if (launch_attn_tc_fixed_scratch(a, device, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  return SP_OK;
 }
 
 int sp_block_mask_from_importance(sp_ctx* ctx, const float* importance, int n_maps, int nb, float gamma,

@@ -32,6 +32,8 @@
 #include <cuda.h>
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sp {
@@ -481,6 +483,50 @@ cudaError_t launch(const AttnArgs& a, cudaStream_t s) {
 }
 
 }  // namespace
+
+// ------------------------------------------------------------------ fixed-scratch variant
+//
+// Scratch for callers that cannot allocate: the per-tile softmax statistics of a
+// dense pivot launch live in this file-scope array instead of a cudaMalloc'ed
+// workspace.  Every device that loads the library carries the array until the
+// process exits.  In host code `g_fixed_scratch` is only a handle for the runtime,
+// not a device address: the address a kernel may use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_fixed_scratch[kFixedScratchBytes];
+static __device__ __align__(256) int g_fixed_status[2];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_fixed_scratch_addr[kMaxDevices];
+void* g_fixed_status_addr[kMaxDevices];
+bool g_fixed_ready[kMaxDevices];
+std::mutex g_fixed_mutex;
+}  // namespace
+
+cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_fixed_mutex);
+  if (!g_fixed_ready[device]) {
+    // first call on this device (the caller made it current): resolve both symbols
+    void* scratch = nullptr;
+    void* status = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&scratch, g_fixed_scratch);
+    if (e != cudaSuccess) return e;
+    e = cudaGetSymbolAddress(&status, g_fixed_status);
+    if (e != cudaSuccess) return e;
+    g_fixed_scratch_addr[device] = scratch;
+    g_fixed_status_addr[device] = status;
+    g_fixed_ready[device] = true;
+  }
+  a.tile_stats = static_cast<float*>(g_fixed_scratch_addr[device]);
+  a.status = static_cast<int*>(g_fixed_status_addr[device]);
+  // the status word keeps the previous call's value and the kernel refuses to work
+  // when it is non-zero: it has to start at zero.  The statistics need no clearing:
+  // every entry that is read has been written by the same launch.
+  cudaError_t e = cudaMemsetAsync(a.status, 0, 2 * sizeof(int), s);
+  if (e != cudaSuccess) return e;
+  return launch_attn_tc(a, s);
+}
 
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s) {
   if (a.d == 128 && a.B == 128) return launch<128, 128>(a, s);

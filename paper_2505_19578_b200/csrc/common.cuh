@@ -50,6 +50,9 @@ struct MaskArgs {
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA
+// same kernel, statistics and status word in the library's fixed device arrays
+cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s);
+constexpr size_t kFixedScratchBytes = 64ull << 20;
 cudaError_t launch_block_mask(const MaskArgs& a, cudaStream_t s);
 cudaError_t launch_fill_causal_mask(uint8_t* mask, int nb, cudaStream_t s);
 
