@@ -306,8 +306,9 @@ def run_ours(args):
         ctx.sp_prefill_attn(dq, dk, dv, cm, piv, gamma, B, out, mask_out=None, stream=stream)
         hout.copy_(out, non_blocking=True)
 
-    e2e_steps = max(1, min(args.steps, 5))
-    e2e_step()
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 5))
+    if e2e_steps:
+        e2e_step()
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record(stream)
@@ -315,7 +316,7 @@ def run_ours(args):
         e2e_step()
     f1.record(stream)
     barrier()
-    e2e_ms_local = f0.elapsed_time(f1) / e2e_steps
+    e2e_ms_local = f0.elapsed_time(f1) / e2e_steps if e2e_steps else float("nan")
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
     d2h = hout.numel() * hout.element_size()
 
@@ -398,6 +399,7 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
