@@ -55,3 +55,56 @@ def compare_mask_rows(gpu_mask, ref_mask, infos, gamma, rows, band=MASK_BAND):
         else:
             bad += 1
     return bad, exempt
+
+
+# ------------------------------------------------------------------ whole-layer helpers
+
+def run_layer(binding, L, gamma, kernel, row_blocks=None):
+    cfg = L["cfg"]
+    ctx = binding.Context(kernel=kernel)
+    qd, kd, vd = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+    Nb = cfg.seq // cfg.block
+    out = torch.full_like(qd, float("nan"))
+    mask = torch.full((cfg.n_q_heads, Nb, Nb), 9, dtype=torch.uint8, device="cuda")
+    ctx.sp_prefill_attn(qd, kd, vd, L["cluster_map"], L["pivot_heads"], gamma, cfg.block, out, mask_out=mask)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    return out, mask
+
+
+def check_layer(L, gamma, out, mask, row_blocks=None):
+    cfg = L["cfg"]
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    Q, K, V = f64(L["q"]), f64(L["k"]), f64(L["v"])
+    g = gamma32(gamma)
+    rows = list(range(Nb)) if row_blocks is None else row_blocks
+    ref = orc.prefill_attn(Q, K, V, L["cluster_map"], L["pivot_heads"], g, B, row_blocks=row_blocks)
+    mask_np = mask.cpu().numpy()
+    bad = exempt = 0
+    src, mask_src = orc.share_masks(L["cluster_map"], L["pivot_heads"])
+    clean_pivot = {}
+    for t, p in enumerate(L["pivot_heads"]):
+        b, e = compare_mask_rows(mask_np[p], ref["mask"][p], ref["infos"][t], g, rows)
+        bad += b
+        exempt += e
+        clean_pivot[t] = {i for i in rows if np.array_equal(mask_np[p][i], ref["mask"][p][i])}
+    assert bad == 0, f"{bad} row-blocks differ outside the {MASK_BAND} band ({exempt} inside)"
+    worst = (0.0, 0.0)
+    for h in range(cfg.n_q_heads):
+        # members report their pivot's mask, dense heads the causal mask
+        if mask_src[h] >= 0:
+            assert np.array_equal(mask_np[h][rows], mask_np[L["pivot_heads"][mask_src[h]]][rows])
+        else:
+            assert np.array_equal(mask_np[h][rows], np.tril(np.ones((Nb, Nb), np.uint8))[rows])
+        assert np.all(np.triu(mask_np[h], 1) == 0)
+        got = f64(out[h])
+        for i in rows:
+            if src[h] >= 0 and i not in clean_pivot[src[h]]:
+                continue                                         # row-block whose mask legitimately flipped
+            sl = slice(i * B, (i + 1) * B)
+            ma, rl = out_errors(got[sl], ref["out"][h][sl])
+            worst = (max(worst[0], ma), max(worst[1], rl))
+    assert worst[0] <= OUT_MAX_ABS and worst[1] <= OUT_REL_L2, worst
+    return worst, exempt
+
+

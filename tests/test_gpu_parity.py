@@ -176,52 +176,8 @@ def test_block_sparse_attn_matches_oracle(binding, kernel, Hq, Hkv, N, d, B):
 
 # ------------------------------------------------------------------ the whole layer
 
-def _run_layer(binding, L, gamma, kernel, row_blocks=None):
-    cfg = L["cfg"]
-    ctx = binding.Context(kernel=kernel)
-    qd, kd, vd = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
-    Nb = cfg.seq // cfg.block
-    out = torch.full_like(qd, float("nan"))
-    mask = torch.full((cfg.n_q_heads, Nb, Nb), 9, dtype=torch.uint8, device="cuda")
-    ctx.sp_prefill_attn(qd, kd, vd, L["cluster_map"], L["pivot_heads"], gamma, cfg.block, out, mask_out=mask)
-    _sync_ok(ctx)
-    return out, mask
-
-
-def _check_layer(L, gamma, out, mask, row_blocks=None):
-    cfg = L["cfg"]
-    B, Nb = cfg.block, cfg.seq // cfg.block
-    Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
-    g = par.gamma32(gamma)
-    rows = list(range(Nb)) if row_blocks is None else row_blocks
-    ref = orc.prefill_attn(Q, K, V, L["cluster_map"], L["pivot_heads"], g, B, row_blocks=row_blocks)
-    mask_np = mask.cpu().numpy()
-    bad = exempt = 0
-    src, mask_src = orc.share_masks(L["cluster_map"], L["pivot_heads"])
-    clean_pivot = {}
-    for t, p in enumerate(L["pivot_heads"]):
-        b, e = par.compare_mask_rows(mask_np[p], ref["mask"][p], ref["infos"][t], g, rows)
-        bad += b
-        exempt += e
-        clean_pivot[t] = {i for i in rows if np.array_equal(mask_np[p][i], ref["mask"][p][i])}
-    assert bad == 0, f"{bad} row-blocks differ outside the {par.MASK_BAND} band ({exempt} inside)"
-    worst = (0.0, 0.0)
-    for h in range(cfg.n_q_heads):
-        # members report their pivot's mask, dense heads the causal mask
-        if mask_src[h] >= 0:
-            assert np.array_equal(mask_np[h][rows], mask_np[L["pivot_heads"][mask_src[h]]][rows])
-        else:
-            assert np.array_equal(mask_np[h][rows], np.tril(np.ones((Nb, Nb), np.uint8))[rows])
-        assert np.all(np.triu(mask_np[h], 1) == 0)
-        got = par.f64(out[h])
-        for i in rows:
-            if src[h] >= 0 and i not in clean_pivot[src[h]]:
-                continue                                         # row-block whose mask legitimately flipped
-            sl = slice(i * B, (i + 1) * B)
-            ma, rl = par.out_errors(got[sl], ref["out"][h][sl])
-            worst = (max(worst[0], ma), max(worst[1], rl))
-    assert worst[0] <= par.OUT_MAX_ABS and worst[1] <= par.OUT_REL_L2, worst
-    return worst, exempt
+_run_layer = par.run_layer
+_check_layer = par.check_layer
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
