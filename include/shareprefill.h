@@ -217,6 +217,19 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
  * kernel kept as an independent on-device cross-check. */
 int sp_ctx_set_kernel(sp_ctx* ctx, int which);
 
+/* Phase trace of the tensor-core attention kernel (a profiling aid).  While a
+ * buffer is set, the CTA that owns the longest row-block of the first listed head
+ * of every attention launch records, for each of its three roles (0 = TMA
+ * producer, 1 = MMA issuer, 2 = softmax thread 0), up to `events_per_role`
+ * pairs {(event_id << 32) | step, SM clock} into
+ * events[(role * events_per_role + n) * 2 .. +1].  Event ids: 20/21 K/V load
+ * issued; 1 K tile landed, 2 QK^T issued, 3 P and V ready, 4 PV issued; 10 S
+ * ready, 11 S in registers, 12 row max done, 13 exponentials done, 14 O
+ * rescaled, 15 P stored and signalled.  `events` is a device buffer of
+ * 3 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
+ * switches tracing off. */
+int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
+
 /* Number of kernels this context has launched since creation (for callers
  * that account for launches). */
 int64_t sp_ctx_launch_count(const sp_ctx* ctx);

@@ -29,6 +29,7 @@ EXPORTS = (
     "sp_ctx_create", "sp_ctx_destroy", "sp_workspace_bytes", "sp_ctx_reserve", "sp_get_status",
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
+    "sp_ctx_set_trace",
 )
 
 
@@ -71,6 +72,7 @@ def load() -> ctypes.CDLL:
     lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
     lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
+    lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
     lib.sp_ctx_launch_count.restype = ctypes.c_int64
     for name in EXPORTS:
@@ -138,6 +140,11 @@ class Context:
 
     def set_kernel(self, kernel: str):
         _check(self._lib.sp_ctx_set_kernel(self._h, {"tc": 0, "simt": 1}[kernel]), "sp_ctx_set_kernel")
+
+    def set_trace(self, events, events_per_role: int):
+        """events: zeroed CUDA int64 tensor of 3 * events_per_role * 2 entries, or None to switch off."""
+        _check(self._lib.sp_ctx_set_trace(self._h, _ptr(events), events_per_role if events is not None else 0),
+               "sp_ctx_set_trace")
 
     def launch_count(self) -> int:
         return int(self._lib.sp_ctx_launch_count(self._h))

@@ -16,6 +16,8 @@ struct sp_ctx {
   int* status = nullptr;  // device int[2]
   int kernel = 0;         // 0 tensor-core, 1 CUDA-core cross-check
   int64_t launches = 0;
+  long long* trace = nullptr;  // caller's device buffer for the phase trace, or null
+  int trace_cap = 0;
 };
 
 namespace {
@@ -91,6 +93,8 @@ AttnArgs base_args(const sp_ctx* ctx, const Problem& p, const sp_tensor* q, cons
   a.n_q_heads = p.Hq; a.n_kv_heads = p.Hkv;
   a.N = p.N; a.d = p.d; a.B = p.B; a.Nb = p.Nb; a.group = p.Hq / p.Hkv;
   a.status = ctx->status;
+  a.trace = ctx->trace;
+  a.trace_cap = ctx->trace_cap;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.d));
   return a;
 }
@@ -233,6 +237,13 @@ int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
 }
 
 int64_t sp_ctx_launch_count(const sp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role) {
+  if (!ctx || events_per_role < 0 || (events_per_role > 0 && !events)) return SP_ERR_INVALID_ARG;
+  ctx->trace = events_per_role > 0 ? reinterpret_cast<long long*>(events) : nullptr;
+  ctx->trace_cap = events_per_role;
+  return SP_OK;
+}
 
 int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v, const int32_t* heads,
                         int n_heads, int block, sp_tensor* out, float* importance_out, float* lse_out, void* stream) {

@@ -229,6 +229,17 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
   const int32_t* idx = list >= 0 ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;
   const bool emit = a.importance != nullptr && list < 0;
   const Abort ab{abort_flag, a.status};
+  // Optional phase trace (one CTA, one thread per role): {(event << 32) | tile, SM clock} pairs.
+  const bool tracing = a.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  int trace_n = 0;
+  auto trace = [&](int role, int event, int tile) {
+    if (tracing && trace_n < a.trace_cap) {
+      long long* e = a.trace + ((size_t)role * a.trace_cap + trace_n) * 2;
+      e[0] = ((long long)event << 32) | (unsigned)tile;
+      e[1] = clock64();
+      ++trace_n;
+    }
+  };
 
   if (threadIdx.x == 0) {
     mbar_init(bar(BAR_Q_FULL), 1);
@@ -268,11 +279,13 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
         mbar_expect_tx(bar(BAR_K_FULL), P::KV_TX);
         for (int b = 0; b < P::NBOX; ++b) tma_load_3d(sK + b * P::KBOX, &tm_k, bar(BAR_K_FULL), b * 64, j * BLK, g);
         ++issued_k;
+        trace(0, 20, t);
         if (t > 0) ok = mbar_wait(bar(BAR_PV_DONE), (t - 1) & 1, ab, 11);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_V_FULL), P::KV_TX);
         for (int b = 0; b < P::NBOX; ++b) tma_load_3d(sV + b * P::KBOX, &tm_v, bar(BAR_V_FULL), b * 64, j * BLK, g);
         ++issued_v;
+        trace(0, 21, t);
       }
       if (*abort_flag) {
         // let the copies already in flight land before the CTA gives its shared memory back
@@ -295,6 +308,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
+        trace(1, 1, t);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk >> 2) * P::QBOX + (kk & 3) * 32;
@@ -302,12 +316,14 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
           mma_ss(tmem + P::S_COL, smem_desc(sQ + off, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, kk > 0);
         }
         mma_commit(bar(BAR_QK_DONE));
+        trace(1, 2, t);
       }
       __syncwarp();
       ok = mbar_wait(bar(BAR_P_FULL), t & 1, ab, 22) && mbar_wait(bar(BAR_V_FULL), t & 1, ab, 23);
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) {
+        trace(1, 3, t);
 #pragma unroll
         for (int kk = 0; kk < BLK / 16; ++kk) {
           // V tile: rows = keys (the MMA's K), 128-byte rows of 64 head-dim columns per box (N-major)
@@ -315,6 +331,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
                  (t > 0 || kk > 0) ? 1u : 0u);
         }
         mma_commit(bar(BAR_PV_DONE));
+        trace(1, 4, t);
       }
       __syncwarp();
     }
@@ -334,9 +351,11 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
       ok = mbar_wait(bar(BAR_QK_DONE), t & 1, ab, 30);
       if (!ok) break;
       tc_fence_after();
+      if (threadIdx.x == 0) trace(2, 10, t);
       uint32_t s[BLK];
 #pragma unroll
       for (int c = 0; c < BLK / 32; ++c) tmem_ld32(tl + P::S_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      if (threadIdx.x == 0) trace(2, 11, t);
       float mx = -CUDART_INF_F;
       if (j == i) {
 #pragma unroll
@@ -350,6 +369,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
         for (int c = 0; c < BLK; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
       }
       mx *= scale;
+      if (threadIdx.x == 0) trace(2, 12, t);
       // the reference max only moves when the row max has grown by more than 2^8
       const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
       const float alpha = ex2_approx(m_ref - m_new);
@@ -363,6 +383,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
         p[c / 2] = pack_bf16(p0, p1);
       }
       l = l * alpha + sum;
+      if (threadIdx.x == 0) trace(2, 13, t);
       if (emit && row_valid) stats[(size_t)t * BLK + row] = m_new + log2f(sum);
       if (t > 0 && __any_sync(0xffffffffu, m_new != m_ref)) {
         // O of the previous steps is relative to the old reference: bring it to the new one
@@ -376,11 +397,13 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
         }
       }
       m_ref = m_new;
+      if (threadIdx.x == 0) trace(2, 14, t);
 #pragma unroll
       for (int c = 0; c < BLK / 64; ++c) tmem_st32(tl + P::S_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p[c * 32]));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL));
+      if (threadIdx.x == 0) trace(2, 15, t);
     }
     if (ok) ok = mbar_wait(bar(BAR_PV_DONE), (cnt - 1) & 1, ab, 31);
     if (ok) {
