@@ -212,21 +212,25 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
                     const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
                     float gamma, int block, sp_tensor* out, uint8_t* mask_out, void* stream);
 
-/* Which attention kernel the context launches: 0 = tensor-core kernel
- * (tcgen05 / TMEM / TMA; the product path, default), 1 = plain fp32 CUDA-core
- * kernel kept as an independent on-device cross-check. */
+/* Which attention kernel the context launches: 0 = tensor-core kernels
+ * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
+ * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V
+ * tiles, otherwise the one-row-block kernel), 1 = plain fp32 CUDA-core kernel
+ * kept as an independent on-device cross-check, 2 = the one-row-block
+ * tensor-core kernel for every shape. */
 int sp_ctx_set_kernel(sp_ctx* ctx, int which);
 
-/* Phase trace of the tensor-core attention kernel (a profiling aid).  While a
- * buffer is set, the CTA that owns the longest row-block of the first listed head
- * of every attention launch records, for each of its three roles (0 = TMA
- * producer, 1 = MMA issuer, 2 = softmax thread 0), up to `events_per_role`
+/* Phase trace of the tensor-core attention kernels (a profiling aid).  While a
+ * buffer is set, the CTA that owns the longest row-block(s) of the first listed
+ * head of every attention launch records, for each of its roles (0 = TMA
+ * producer, 1 = MMA issuer, 2 = softmax thread 0 of the first row-block, 3 = the
+ * same of the second row-block, paired kernel only), up to `events_per_role`
  * pairs {(event_id << 32) | step, SM clock} into
  * events[(role * events_per_role + n) * 2 .. +1].  Event ids: 20/21 K/V load
  * issued; 1 K tile landed, 2 QK^T issued, 3 P and V ready, 4 PV issued; 10 S
  * ready, 11 S in registers, 12 row max done, 13 exponentials done, 14 O
  * rescaled, 15 P stored and signalled.  `events` is a device buffer of
- * 3 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
+ * 4 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
  * switches tracing off. */
 int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
 

@@ -14,7 +14,7 @@ struct sp_ctx {
   void* ws = nullptr;
   size_t ws_bytes = 0;
   int* status = nullptr;  // device int[2]
-  int kernel = 0;         // 0 tensor-core, 1 CUDA-core cross-check
+  int kernel = 0;         // 0 tensor-core (paired where supported), 1 CUDA-core cross-check, 2 tensor-core single-tile
   int64_t launches = 0;
   long long* trace = nullptr;  // caller's device buffer for the phase trace, or null
   int trace_cap = 0;
@@ -119,7 +119,10 @@ int reserve(sp_ctx* ctx, size_t bytes) {
 
 int launch_attn(sp_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   if (a.n_heads == 0) return SP_OK;
-  cudaError_t e = ctx->kernel == 1 ? launch_attn_simt(a, s) : launch_attn_tc(a, s);
+  cudaError_t e;
+  if (ctx->kernel == 1) e = launch_attn_simt(a, s);
+  else if (ctx->kernel == 0 && attn_pair_supported(a)) e = launch_attn_pair(a, s);
+  else e = launch_attn_tc(a, s);
   if (e != cudaSuccess) return SP_ERR_CUDA;
   ctx->launches += 1;
   return SP_OK;
@@ -231,7 +234,7 @@ int sp_get_status(sp_ctx* ctx, int* code, int* where) {
 }
 
 int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
-  if (!ctx || (which != 0 && which != 1)) return SP_ERR_INVALID_ARG;
+  if (!ctx || which < 0 || which > 2) return SP_ERR_INVALID_ARG;
   ctx->kernel = which;
   return SP_OK;
 }
@@ -262,7 +265,7 @@ int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, con
   for (int t = 0; t < n_heads; ++t) { a.heads.v[t] = heads[t]; a.lists.v[t] = -1; }
   a.importance = importance_out;
   a.lse = lse_out;
-  if (importance_out && ctx->kernel == 0) {
+  if (importance_out && ctx->kernel != 1) {
     if ((rc = reserve(ctx, align_up((size_t)n_heads * tile_stats_bytes_per_head(p.Nb, p.B))))) return rc;
     a.tile_stats = static_cast<float*>(ctx->ws);
   }

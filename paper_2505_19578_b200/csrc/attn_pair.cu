@@ -1,0 +1,557 @@
+// Paired-row-block tensor-core attention kernel for sm_100a (head_dim 128,
+// block 128): dense (pivot) and block-sparse (member) causal attention.
+//
+//   Section 5.1:  O = softmax(Q K^T / sqrt(d) - c (1 - M)) V,  c -> infinity,
+//   causal.  A pivot walks every causal key-block and also emits the softmax
+//   probability mass of each (query-block, key-block) tile; a member walks the
+//   compacted list of key-blocks its cluster's pivot selected.
+//
+// One CTA owns one head and TWO adjacent query row-blocks (tile A = row-block
+// 2u, tile B = row-block 2u+1), 256 query rows, and occupies a whole SM.  The
+// two tiles walk the UNION of their key-block lists in ascending order, so a
+// K/V tile both of them need is brought into shared memory once and feeds four
+// MMAs instead of two; a key-block only one of them selected is computed for
+// that tile alone.  (Dense: the union is 0..2u+1, the last key-block is B's
+// diagonal tile only.)
+//
+// Warp roles (384 threads):
+//   warps 0-3   softmax of tile A: thread t owns query row t = TMEM lane t
+//   warps 4-7   softmax of tile B
+//   warp  8     MMA issuer, owner of the TMEM allocation (all 512 columns:
+//               S_A, S_B, O_A, O_B, 128 fp32 columns each)
+//   warp  9     producer: merges the two lists, TMA loads of Q (once) and of
+//               the K and V tiles into two-stage rings (128-byte swizzle)
+//   warps 10-11 idle (they only give their registers to the softmax warps)
+//
+// Order of the MMAs, per merged key-block n:  PV_A(n), QK_A(n+1), PV_B(n),
+// QK_B(n+1).  While the softmax warps of A work on S_A(n) the tensor pipe runs
+// PV_B(n-1) and QK_B(n); while those of B work on S_B(n) it runs PV_A(n) and
+// QK_A(n+1).  P (bf16) overwrites the first half of the S columns it came from
+// and is the TMEM A operand of PV; the next QK of that tile is issued after the
+// PV that reads P, and the tensor pipe keeps issue order.
+//
+// Block importance in one pass: as in the single-tile kernel, each softmax
+// thread spills one float per visited tile, stat = m + log2(sum_c 2^(s_c - m))
+// with m the row's reference max at that step; after the last tile the row's
+// log-sum-exp L is known and the tile mass is (1/B) sum_rows 2^(stat - L).
+//
+// Every wait on an mbarrier is bounded: when it runs out the CTA raises an abort
+// flag, records SP_ERR_TIMEOUT in the status word, and all roles fall through
+// to the common teardown (TMEM is freed, the kernel returns).
+#include "tc_ptx.cuh"
+
+namespace sp {
+namespace {
+
+using namespace tc;
+
+constexpr int D = 128;      // head_dim
+constexpr int BLK = 128;    // block
+constexpr int kThreadsPair = 384;
+constexpr int kStages = 2;  // K ring and V ring depth
+
+// shared-memory plan (bytes)
+constexpr int kBox = 128 * 128;                 // one 64-column box of 128 rows
+constexpr int kTile = 2 * kBox;                 // a 128 x 128 bf16 tile (two boxes)
+constexpr int kQOff = 0;                        // [box][tile A|B][128 rows][128 B]
+constexpr int kKOff = kQOff + 2 * kTile;        // [stage][box][128 rows][128 B]
+constexpr int kVOff = kKOff + kStages * kTile;
+constexpr int kMiscOff = kVOff + kStages * kTile;
+constexpr int kMiscBytes = 2048;
+constexpr int kSmemTotal = kMiscOff + kMiscBytes + 1024;   // + slack for 1024-byte alignment
+
+// TMEM columns
+constexpr uint32_t kSCol = 0;      // S_A at 0, S_B at 128 (P reuses the first 64 columns of each)
+constexpr uint32_t kOCol = 256;    // O_A at 256, O_B at 384
+
+enum {
+  BAR_Q_FULL = 0,
+  BAR_K_FULL,                          // + stage
+  BAR_K_EMPTY = BAR_K_FULL + kStages,  // + stage
+  BAR_V_FULL = BAR_K_EMPTY + kStages,
+  BAR_V_EMPTY = BAR_V_FULL + kStages,
+  BAR_S_FULL = BAR_V_EMPTY + kStages,  // + tile (A = 0, B = 1)
+  BAR_P_FULL = BAR_S_FULL + 2,
+  BAR_O_DONE = BAR_P_FULL + 2,
+  BAR_COUNT = BAR_O_DONE + 2
+};
+
+enum { F_A = 1, F_B = 2, F_LAST = 4 };
+
+// ------------------------------------------------------------------ small PTX helpers of this kernel
+
+__device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+// Waits for this thread's outstanding tcgen05.ld and pins the 32 registers behind the wait,
+// so that nothing that reads them can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void reg_fence32(uint32_t* r) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])::"memory");
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// (d0, d1) = (a0, a1) * (b, b) + (c, c): one packed FMA
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
+  asm("{\n\t.reg .b64 ra, rd;\n\t"
+      "mov.b64 rd, {%0, %1};\n\tmov.b64 ra, {%2, %3};\n\t"
+      "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(d0), "+f"(d1)
+      : "f"(a0), "f"(a1));
+}
+// bf16x2 with `lo` in the low half
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+template <int N>
+__device__ __forceinline__ void set_regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void set_regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// One tile's geometry as seen by every role.
+struct TileInfo {
+  int i;                 // row-block
+  int cnt;               // key-blocks it visits
+  const int32_t* idx;    // its ascending key-block list, or null = 0..i
+};
+
+__global__ void __launch_bounds__(kThreadsPair, 1)
+attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sQ = smem_u32(smem + kQOff), sK = smem_u32(smem + kKOff), sV = smem_u32(smem + kVOff);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kMiscOff);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kMiscOff + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kMiscOff + 260);
+  volatile int* kflags = reinterpret_cast<volatile int*>(smem + kMiscOff + 264);   // [kStages]
+  float* lse_smem = reinterpret_cast<float*>(smem + kMiscOff + 512);               // [2][128]
+  auto bar = [&](int which) { return smem_u32(bars + which); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_pairs = (a.Nb + 1) >> 1;
+  const int u = n_pairs - 1 - (int)blockIdx.x;      // long row-blocks first
+  const int slot = blockIdx.y;
+  const int h = a.heads.v[slot];
+  const int g = h / a.group;
+  const int list = a.lists.v[slot];
+  const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
+  TileInfo tile[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    const int i = 2 * u + x;
+    int cnt = 0;
+    if (i < a.Nb && !poisoned) {
+      cnt = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
+      cnt = cnt < 0 ? 0 : (cnt > i + 1 ? i + 1 : cnt);
+    }
+    tile[x].i = i;
+    tile[x].cnt = cnt;
+    tile[x].idx = list >= 0 ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;
+  }
+  const bool any_work = tile[0].cnt + tile[1].cnt > 0;
+  const bool emit = a.importance != nullptr && list < 0;
+  const Abort ab{abort_flag, a.status};
+  // Optional phase trace (one CTA, one thread per role): {(event << 32) | step, SM clock} pairs.
+  const bool tracing = a.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  int trace_n = 0;
+  auto trace = [&](int role, int event, int step) {
+    if (tracing && trace_n < a.trace_cap) {
+      long long* e = a.trace + ((size_t)role * a.trace_cap + trace_n) * 2;
+      e[0] = ((long long)event << 32) | (unsigned)step;
+      e[1] = clock64();
+      ++trace_n;
+    }
+  };
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(BAR_Q_FULL), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(BAR_K_FULL + s), 1);
+      mbar_init(bar(BAR_K_EMPTY + s), 1);
+      mbar_init(bar(BAR_V_FULL + s), 1);
+      mbar_init(bar(BAR_V_EMPTY + s), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar(BAR_S_FULL + x), 1);
+      mbar_init(bar(BAR_P_FULL + x), 128);
+      mbar_init(bar(BAR_O_DONE + x), 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) tmem_alloc(smem_u32(tmem_slot), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp >= 8) {
+    set_regs_dec<64>();
+    if (warp == 9) {
+      // ---------------------------------------------------------- producer
+      if (any_work) {
+        if (lane == 0) {
+          const int n_q = tile[1].i < a.Nb ? 2 : 1;
+          mbar_expect_tx(bar(BAR_Q_FULL), n_q * kTile);
+          for (int x = 0; x < n_q; ++x)
+            for (int b = 0; b < 2; ++b)
+              tma_load_3d(sQ + b * kTile + x * kBox, &tm_q, bar(BAR_Q_FULL), b * 64, tile[x].i * BLK, h);
+        }
+        // The two ascending lists are merged 32 entries at a time: lane l holds entry base + l.
+        const int cntA = tile[0].cnt, cntB = tile[1].cnt;
+        const int32_t* idxA = tile[0].idx;
+        const int32_t* idxB = tile[1].idx;
+        int pa = 0, pb = 0, n = 0, issued_k = 0, issued_v = 0;
+        int chunkA = 0, chunkB = 0;
+        if (idxA) chunkA = lane < cntA ? idxA[lane] : 0;
+        if (idxB) chunkB = lane < cntB ? idxB[lane] : 0;
+        bool ok = true;
+        while ((pa < cntA || pb < cntB) && ok) {
+          const int ja = pa < cntA ? (idxA ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
+          const int jb = pb < cntB ? (idxB ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
+          const int j = ja < jb ? ja : jb;
+          int f = (ja == j ? F_A : 0) | (jb == j ? F_B : 0);
+          if (ja == j) {
+            ++pa;
+            if (idxA && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
+          }
+          if (jb == j) {
+            ++pb;
+            if (idxB && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
+          }
+          if (!(pa < cntA || pb < cntB)) f |= F_LAST;
+          const int st = n % kStages;
+          const uint32_t ph = (uint32_t)(n / kStages) & 1u;
+          if (n >= kStages) ok = mbar_wait(bar(BAR_K_EMPTY + st), ph ^ 1u, ab, 10);
+          if (!ok) break;
+          if (lane == 0) {
+            kflags[st] = f;
+            mbar_expect_tx(bar(BAR_K_FULL + st), kTile);
+            for (int b = 0; b < 2; ++b) tma_load_3d(sK + st * kTile + b * kBox, &tm_k, bar(BAR_K_FULL + st), b * 64, j * BLK, g);
+            trace(0, 20, n);
+          }
+          ++issued_k;
+          if (n >= kStages) ok = mbar_wait(bar(BAR_V_EMPTY + st), ph ^ 1u, ab, 11);
+          if (!ok) break;
+          if (lane == 0) {
+            mbar_expect_tx(bar(BAR_V_FULL + st), kTile);
+            for (int b = 0; b < 2; ++b) tma_load_3d(sV + st * kTile + b * kBox, &tm_v, bar(BAR_V_FULL + st), b * 64, j * BLK, g);
+            trace(0, 21, n);
+          }
+          ++issued_v;
+          ++n;
+        }
+        if (*abort_flag && lane == 0) {
+          // let the copies already in flight land before the CTA gives its shared memory back
+          const long long t0 = clock64();
+          while (clock64() - t0 < kWaitCycles / 8) {
+            bool done = mbar_try_wait(bar(BAR_Q_FULL), 0);
+            for (int back = 1; back <= kStages; ++back) {   // at most the last kStages loads of a ring are in flight
+              const int mk = issued_k - back, mv = issued_v - back;
+              if (mk >= 0) done = done && mbar_try_wait(bar(BAR_K_FULL + mk % kStages), (uint32_t)(mk / kStages) & 1u);
+              if (mv >= 0) done = done && mbar_try_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u);
+            }
+            if (done) break;
+          }
+        }
+      }
+    } else if (warp == 8) {
+      // ---------------------------------------------------------- MMA issuer
+      constexpr uint32_t idesc_qk = instr_desc(128, BLK, 0, 0);
+      constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
+      const int cntA = tile[0].cnt, cntB = tile[1].cnt;
+      auto issue_qk = [&](int x, int st) {     // S_x = Q_x K^T from K stage st
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t qoff = (kk >> 2) * kTile + x * kBox + (kk & 3) * 32;
+          const uint32_t koff = st * kTile + (kk >> 2) * kBox + (kk & 3) * 32;
+          mma_ss(tmem + kSCol + x * 128, smem_desc(sQ + qoff, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, kk > 0);
+        }
+        mma_commit(bar(BAR_S_FULL + x));
+      };
+      auto issue_pv = [&](int x, int st, bool accumulate) {   // O_x (+)= P_x V from V stage st
+#pragma unroll
+        for (int kk = 0; kk < BLK / 16; ++kk) {
+          // V tile: rows = keys (the MMA's K), 128-byte rows of 64 head-dim columns per box (N-major)
+          mma_ts(tmem + kOCol + x * 128, tmem + kSCol + x * 128 + kk * 8,
+                 smem_desc(sV + st * kTile + kk * 16 * 128, kBox, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+        }
+      };
+      bool ok = any_work ? mbar_wait(bar(BAR_Q_FULL), 0, ab, 20) : false;
+      if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, ab, 21);
+      int f = 0, n = 0, tA = 0, tB = 0;
+      if (ok) {
+        tc_fence_after();
+        f = kflags[0];
+        if (lane == 0) {
+          trace(1, 1, 0);
+          if (f & F_A) issue_qk(0, 0);
+          if (f & F_B) issue_qk(1, 0);
+          mma_commit(bar(BAR_K_EMPTY + 0));
+          trace(1, 2, 0);
+        }
+        __syncwarp();
+      }
+      while (ok) {
+        const bool last = (f & F_LAST) != 0;
+        const int st = n % kStages, stn = (n + 1) % kStages;
+        const uint32_t ph = (uint32_t)(n / kStages) & 1u, phn = (uint32_t)((n + 1) / kStages) & 1u;
+        int fn = 0;
+        if (!last) {
+          ok = mbar_wait(bar(BAR_K_FULL + stn), phn, ab, 22);
+          if (!ok) break;
+          fn = kflags[stn];
+        }
+        ok = mbar_wait(bar(BAR_V_FULL + st), ph, ab, 23);
+        if (!ok) break;
+        if (f & F_A) {
+          ok = mbar_wait(bar(BAR_P_FULL + 0), tA & 1, ab, 24);
+          if (!ok) break;
+        }
+        tc_fence_after();
+        if (lane == 0) {
+          trace(1, 3, n);
+          if (f & F_A) {
+            issue_pv(0, st, tA > 0);
+            if (tA + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
+          }
+          if (fn & F_A) issue_qk(0, stn);
+        }
+        __syncwarp();
+        if (f & F_A) ++tA;
+        if (f & F_B) {
+          ok = mbar_wait(bar(BAR_P_FULL + 1), tB & 1, ab, 25);
+          if (!ok) break;
+        }
+        tc_fence_after();
+        if (lane == 0) {
+          if (f & F_B) {
+            issue_pv(1, st, tB > 0);
+            if (tB + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
+          }
+          mma_commit(bar(BAR_V_EMPTY + st));
+          if (fn & F_B) issue_qk(1, stn);
+          if (!last) mma_commit(bar(BAR_K_EMPTY + stn));
+          trace(1, 4, n);
+        }
+        __syncwarp();
+        if (f & F_B) ++tB;
+        if (last) break;
+        f = fn;
+        ++n;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue of tile x
+    set_regs_inc<216>();
+    const int x = warp >> 2;
+    const int row = threadIdx.x & 127;                 // TMEM lane == query row inside the tile
+    const int i = x ? tile[1].i : tile[0].i, cnt = x ? tile[1].cnt : tile[0].cnt;
+    const int32_t* idx = x ? tile[1].idx : tile[0].idx;
+    const int r = i * BLK + row;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t tS = tl + kSCol + x * 128, tO = tl + kOCol + x * 128;
+    const float scale = a.scale_log2;
+    const int trole = 2 + x;
+    const bool tthread = row == 0;
+    float* stats = emit ? a.tile_stats + ((size_t)slot * ((size_t)a.Nb * (a.Nb + 1) / 2) + (size_t)i * (i + 1) / 2) * BLK
+                        : nullptr;
+    float m_ref = -CUDART_INF_F, l = 0.f;
+    bool ok = cnt > 0;
+    int j_next = cnt > 0 ? (idx ? idx[0] : 0) : 0;
+    for (int t = 0; t < cnt && ok; ++t) {
+      const int j = j_next;
+      if (t + 1 < cnt) j_next = idx ? idx[t + 1] : t + 1;
+      ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, ab, 30 + x);
+      if (!ok) break;
+      tc_fence_after();
+      if (tthread) trace(trole, 10, t);
+      uint32_t s[BLK];
+#pragma unroll
+      for (int c = 0; c < BLK / 32; ++c) tmem_ld32_async(tS + c * 32, &s[c * 32]);
+      tmem_ld_wait();
+#pragma unroll
+      for (int c = 0; c < BLK / 32; ++c) reg_fence32(&s[c * 32]);
+      if (tthread) trace(trole, 11, t);
+      if (j == i) {
+#pragma unroll
+        for (int c = 0; c < BLK; ++c)
+          if (c > row) s[c] = __float_as_uint(-CUDART_INF_F);
+      }
+      float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[1]));
+      float mx1 = fmaxf(__uint_as_float(s[2]), __uint_as_float(s[3]));
+      float mx2 = fmaxf(__uint_as_float(s[4]), __uint_as_float(s[5]));
+      float mx3 = fmaxf(__uint_as_float(s[6]), __uint_as_float(s[7]));
+#pragma unroll
+      for (int c = 8; c < BLK; c += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[c + 0]), __uint_as_float(s[c + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
+      if (tthread) trace(trole, 12, t);
+      // the reference max only moves when the row max has grown by more than 2^8
+      const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+      const float alpha = ex2_approx(m_ref - m_new);
+      const float neg_m = -m_new;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+      uint32_t p[BLK / 2];
+#pragma unroll
+      for (int c = 0; c < BLK; c += 4) {
+        float x0, x1, x2, x3;
+        fma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), scale, neg_m);
+        fma2(x2, x3, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]), scale, neg_m);
+        x0 = ex2_approx(x0);
+        x1 = ex2_approx(x1);
+        x2 = ex2_approx(x2);
+        x3 = ex2_approx(x3);
+        add2(sum0, sum1, x0, x1);
+        add2(sum2, sum3, x2, x3);
+        p[c / 2] = cvt_bf16x2(x0, x1);
+        p[c / 2 + 1] = cvt_bf16x2(x2, x3);
+      }
+      const float sum = (sum0 + sum1) + (sum2 + sum3);
+      l = l * alpha + sum;
+      if (tthread) trace(trole, 13, t);
+      if (emit) stats[(size_t)t * BLK + row] = m_new + log2f(sum);
+      if (t > 0 && __any_sync(0xffffffffu, m_new != m_ref)) {
+        // O of the previous steps is relative to the old reference: bring it to the new one.
+        // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + c * 32, o);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(tO + c * 32, o);
+        }
+      }
+      m_ref = m_new;
+      if (tthread) trace(trole, 14, t);
+#pragma unroll
+      for (int c = 0; c < BLK / 64; ++c) tmem_st32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p[c * 32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_P_FULL + x));
+      if (tthread) trace(trole, 15, t);
+    }
+    if (ok) ok = mbar_wait(bar(BAR_O_DONE + x), 0, ab, 32 + x);
+    float lse2 = 0.f;
+    if (ok) {
+      tc_fence_after();
+      const float inv_l = 1.f / l;
+      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tO + c * 32, o);
+        uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          uint4 w;
+          w.x = cvt_bf16x2(__uint_as_float(o[8 * e + 0]) * inv_l, __uint_as_float(o[8 * e + 1]) * inv_l);
+          w.y = cvt_bf16x2(__uint_as_float(o[8 * e + 2]) * inv_l, __uint_as_float(o[8 * e + 3]) * inv_l);
+          w.z = cvt_bf16x2(__uint_as_float(o[8 * e + 4]) * inv_l, __uint_as_float(o[8 * e + 5]) * inv_l);
+          w.w = cvt_bf16x2(__uint_as_float(o[8 * e + 6]) * inv_l, __uint_as_float(o[8 * e + 7]) * inv_l);
+          dst[e] = w;
+        }
+      }
+      lse2 = m_ref + log2f(l);
+      if (a.lse) a.lse[(size_t)slot * a.N + r] = lse2 * 0.6931471805599453f;
+    }
+    if (emit) {
+      float* lse_x = lse_smem + x * 128;
+      lse_x[row] = lse2;
+      // the four softmax warps of this tile: statistics and lse visible to one another, and one
+      // common decision (a thread whose wait ran out must not leave the others at a barrier)
+      const bool all_ok = bar_and(1 + x, 128, ok);
+      if (all_ok) {
+        float* imp_row = a.importance + ((size_t)slot * a.Nb + i) * a.Nb;
+        const float4 lse4 = *reinterpret_cast<const float4*>(lse_x + lane * 4);
+        const int wq = warp & 3;
+        // each warp takes tiles wq, wq + 4, ...; eight tiles in flight; lane l sums rows 4l..4l+3
+        for (int t0 = wq; t0 < cnt; t0 += 32) {
+          float4 v[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int t = t0 + 4 * e;
+            v[e] = t < cnt ? *reinterpret_cast<const float4*>(stats + (size_t)t * BLK + lane * 4)
+                           : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            float acc = (ex2_approx(v[e].x - lse4.x) + ex2_approx(v[e].y - lse4.y)) +
+                        (ex2_approx(v[e].z - lse4.z) + ex2_approx(v[e].w - lse4.w));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            const int t = t0 + 4 * e;
+            if (lane == 0 && t < cnt) imp_row[t] = acc * (1.f / BLK);
+          }
+        }
+        for (int jz = i + 1 + row; jz < a.Nb; jz += 128) imp_row[jz] = 0.f;
+      }
+    }
+    if (ok) {
+    } else if (cnt == 0 && i < a.Nb && !poisoned) {
+      // an empty list is outside the contract; leave defined output (zeros) rather than garbage
+      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+      for (int e = 0; e < D / 8; ++e) reinterpret_cast<uint4*>(orow)[e] = make_uint4(0, 0, 0, 0);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+bool attn_pair_supported(const AttnArgs& a) { return a.d == D && a.B == BLK; }
+
+cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s) {
+  if (!attn_pair_supported(a)) return cudaErrorInvalidValue;
+  CUtensorMap tq, tk, tv;
+  if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
+      !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK) ||
+      !make_map(&tv, a.v, a.v_sh, a.v_sn, a.n_kv_heads, a.N, D, BLK))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
+  if (e != cudaSuccess) return e;
+  attn_pair_kernel<<<dim3((a.Nb + 1) / 2, a.n_heads), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
+  return cudaGetLastError();
+}
+
+}  // namespace sp

@@ -35,7 +35,7 @@ struct AttnArgs {
   float* lse;              // [n_heads, N] or null
   float* tile_stats;       // scratch: per (slot, row-block) B floats per causal tile (tensor-core path)
   int* status;             // device int[2]: {code, where}
-  long long* trace;        // optional phase trace of CTA (0,0): 3 roles x trace_cap x {tag, clock}
+  long long* trace;        // optional phase trace of CTA (0,0): 4 roles x trace_cap x {tag, clock}
   int trace_cap;
   float scale_log2;        // log2(e) / sqrt(d)
 };
@@ -51,7 +51,10 @@ struct MaskArgs {
 
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
-cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA, one row-block per CTA
+// tcgen05 / TMEM / TMA, two adjacent row-blocks per CTA sharing their K/V tiles (head_dim 128, block 128)
+bool attn_pair_supported(const AttnArgs& a);
+cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s);
 // same kernel, statistics and status word in the library's fixed device arrays
 cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s);
 constexpr size_t kFixedScratchBytes = 64ull << 20;

@@ -10,7 +10,7 @@ from tests import _parity as par
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = ["tc", "simt"]
+KERNELS = ["tc", "tc1", "simt"]
 
 
 @pytest.fixture(scope="module")
@@ -230,6 +230,7 @@ def test_tc_and_simt_kernels_agree_on_importance(binding):
         _sync_ok(ctx)
         res[kernel] = imp.cpu().numpy()
     np.testing.assert_allclose(res["tc"], res["simt"], rtol=0, atol=par.IMP_ATOL)
+    np.testing.assert_allclose(res["tc1"], res["simt"], rtol=0, atol=par.IMP_ATOL)
 
 
 # ------------------------------------------------------------------ argument checking (host side)
