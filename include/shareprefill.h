@@ -223,14 +223,15 @@ int sp_ctx_set_kernel(sp_ctx* ctx, int which);
 /* Phase trace of the tensor-core attention kernels (a profiling aid).  While a
  * buffer is set, the CTA that owns the longest row-block(s) of the first listed
  * head of every attention launch records, for each of its roles (0 = TMA
- * producer, 1 = MMA issuer, 2 = softmax thread 0 of the first row-block, 3 = the
- * same of the second row-block, paired kernel only), up to `events_per_role`
+ * producer, 1 = MMA issuer (of the first row-block), 2 = softmax thread 0 of the
+ * first row-block; paired kernel only: 3 = softmax thread 0 of the second
+ * row-block, 4 = its MMA issuer), up to `events_per_role`
  * pairs {(event_id << 32) | step, SM clock} into
  * events[(role * events_per_role + n) * 2 .. +1].  Event ids: 20/21 K/V load
  * issued; 1 K tile landed, 2 QK^T issued, 3 P and V ready, 4 PV issued; 10 S
  * ready, 11 S in registers, 12 row max done, 13 exponentials done, 14 O
  * rescaled, 15 P stored and signalled.  `events` is a device buffer of
- * 4 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
+ * 5 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
  * switches tracing off. */
 int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
 

@@ -142,7 +142,7 @@ class Context:
         _check(self._lib.sp_ctx_set_kernel(self._h, {"tc": 0, "simt": 1, "tc1": 2}[kernel]), "sp_ctx_set_kernel")
 
     def set_trace(self, events, events_per_role: int):
-        """events: zeroed CUDA int64 tensor of 4 * events_per_role * 2 entries, or None to switch off."""
+        """events: zeroed CUDA int64 tensor of 5 * events_per_role * 2 entries, or None to switch off."""
         _check(self._lib.sp_ctx_set_trace(self._h, _ptr(events), events_per_role if events is not None else 0),
                "sp_ctx_set_trace")
 

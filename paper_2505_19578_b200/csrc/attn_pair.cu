@@ -24,9 +24,11 @@
 //   warps 10-11 idle (they only give their registers to the softmax warps)
 //
 // Order of the MMAs, per merged key-block n:  PV_A(n), QK_A(n+1), PV_B(n),
-// QK_B(n+1).  While the softmax warps of A work on S_A(n) the tensor pipe runs
-// PV_B(n-1) and QK_B(n); while those of B work on S_B(n) it runs PV_A(n) and
-// QK_A(n+1).  P (bf16) overwrites the first half of the S columns it came from
+// QK_B(n+1), all issued by one thread: while the softmax warps of A work on
+// S_A(n) the tensor pipe runs PV_B(n-1) and QK_B(n); while those of B work on
+// S_B(n) it runs PV_A(n) and QK_A(n+1).  (One issuer per tile was tried: the two
+// tiles then fall into step, their softmax phases coincide and nothing overlaps
+// the MMAs.)  P (bf16) overwrites the first half of the S columns it came from
 // and is the TMEM A operand of PV; the next QK of that tile is issued after the
 // PV that reads P, and the tensor pipe keeps issue order.
 //
@@ -197,8 +199,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(BAR_K_FULL + s), 1);
       mbar_init(bar(BAR_K_EMPTY + s), 1);
-      mbar_init(bar(BAR_V_FULL + s), 1);
       mbar_init(bar(BAR_V_EMPTY + s), 1);
+      mbar_init(bar(BAR_V_FULL + s), 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(BAR_S_FULL + x), 1);
@@ -215,7 +217,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   const uint32_t tmem = *tmem_slot;
 
   if (warp >= 8) {
-    set_regs_dec<64>();
+    set_regs_dec<112>();
     if (warp == 9) {
       // ---------------------------------------------------------- producer
       if (any_work) {
@@ -289,21 +291,28 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       constexpr uint32_t idesc_qk = instr_desc(128, BLK, 0, 0);
       constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
       const int cntA = tile[0].cnt, cntB = tile[1].cnt;
+      // Descriptors differ from these bases only in the 16-byte-unit address field (low word).
+      const uint64_t dq0 = smem_desc(sQ, 16, 1024);
+      const uint64_t dk0 = smem_desc(sK, 16, 1024);
+      const uint64_t dv0 = smem_desc(sV, kBox, 1024);
       auto issue_qk = [&](int x, int st) {     // S_x = Q_x K^T from K stage st
+        const uint64_t dq = dq0 + (uint64_t)((x * kBox) >> 4);
+        const uint64_t dk = dk0 + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t qoff = (kk >> 2) * kTile + x * kBox + (kk & 3) * 32;
-          const uint32_t koff = st * kTile + (kk >> 2) * kBox + (kk & 3) * 32;
-          mma_ss(tmem + kSCol + x * 128, smem_desc(sQ + qoff, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, kk > 0);
+          const uint32_t qoff = ((kk >> 2) * kTile + (kk & 3) * 32) >> 4;
+          const uint32_t koff = ((kk >> 2) * kBox + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + kSCol + x * 128, dq + qoff, dk + koff, idesc_qk, kk > 0);
         }
         mma_commit(bar(BAR_S_FULL + x));
       };
       auto issue_pv = [&](int x, int st, bool accumulate) {   // O_x (+)= P_x V from V stage st
+        const uint64_t dv = dv0 + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
         for (int kk = 0; kk < BLK / 16; ++kk) {
           // V tile: rows = keys (the MMA's K), 128-byte rows of 64 head-dim columns per box (N-major)
-          mma_ts(tmem + kOCol + x * 128, tmem + kSCol + x * 128 + kk * 8,
-                 smem_desc(sV + st * kTile + kk * 16 * 128, kBox, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+          mma_ts(tmem + kOCol + x * 128, tmem + kSCol + x * 128 + kk * 8, dv + (uint32_t)((kk * 16 * 128) >> 4), idesc_pv,
+                 (accumulate || kk > 0) ? 1u : 0u);
         }
       };
       bool ok = any_work ? mbar_wait(bar(BAR_Q_FULL), 0, ab, 20) : false;
@@ -345,6 +354,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
             if (tA + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
           }
           if (fn & F_A) issue_qk(0, stn);
+          trace(1, 5, n);
         }
         __syncwarp();
         if (f & F_A) ++tA;
@@ -354,6 +364,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         tc_fence_after();
         if (lane == 0) {
+          trace(1, 6, n);
           if (f & F_B) {
             issue_pv(1, st, tB > 0);
             if (tB + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
@@ -372,7 +383,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue of tile x
-    set_regs_inc<216>();
+    set_regs_inc<192>();
     const int x = warp >> 2;
     const int row = threadIdx.x & 127;                 // TMEM lane == query row inside the tile
     const int i = x ? tile[1].i : tile[0].i, cnt = x ? tile[1].cnt : tile[0].cnt;
@@ -396,74 +407,103 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       tc_fence_after();
       if (tthread) trace(trole, 10, t);
       uint32_t s[BLK];
+      auto load_s = [&]() {
 #pragma unroll
-      for (int c = 0; c < BLK / 32; ++c) tmem_ld32_async(tS + c * 32, &s[c * 32]);
-      tmem_ld_wait();
+        for (int c = 0; c < BLK / 32; ++c) tmem_ld32_async(tS + c * 32, &s[c * 32]);
+        tmem_ld_wait();
 #pragma unroll
-      for (int c = 0; c < BLK / 32; ++c) reg_fence32(&s[c * 32]);
-      if (tthread) trace(trole, 11, t);
-      if (j == i) {
+        for (int c = 0; c < BLK / 32; ++c) reg_fence32(&s[c * 32]);
+        if (j == i) {
 #pragma unroll
-        for (int c = 0; c < BLK; ++c)
-          if (c > row) s[c] = __float_as_uint(-CUDART_INF_F);
-      }
-      float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[1]));
-      float mx1 = fmaxf(__uint_as_float(s[2]), __uint_as_float(s[3]));
-      float mx2 = fmaxf(__uint_as_float(s[4]), __uint_as_float(s[5]));
-      float mx3 = fmaxf(__uint_as_float(s[6]), __uint_as_float(s[7]));
-#pragma unroll
-      for (int c = 8; c < BLK; c += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[c + 0]), __uint_as_float(s[c + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-      }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
-      if (tthread) trace(trole, 12, t);
-      // the reference max only moves when the row max has grown by more than 2^8
-      const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
-      const float alpha = ex2_approx(m_ref - m_new);
-      const float neg_m = -m_new;
-      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-      uint32_t p[BLK / 2];
-#pragma unroll
-      for (int c = 0; c < BLK; c += 4) {
-        float x0, x1, x2, x3;
-        fma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), scale, neg_m);
-        fma2(x2, x3, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]), scale, neg_m);
-        x0 = ex2_approx(x0);
-        x1 = ex2_approx(x1);
-        x2 = ex2_approx(x2);
-        x3 = ex2_approx(x3);
-        add2(sum0, sum1, x0, x1);
-        add2(sum2, sum3, x2, x3);
-        p[c / 2] = cvt_bf16x2(x0, x1);
-        p[c / 2 + 1] = cvt_bf16x2(x2, x3);
-      }
-      const float sum = (sum0 + sum1) + (sum2 + sum3);
-      l = l * alpha + sum;
-      if (tthread) trace(trole, 13, t);
-      if (emit) stats[(size_t)t * BLK + row] = m_new + log2f(sum);
-      if (t > 0 && __any_sync(0xffffffffu, m_new != m_ref)) {
-        // O of the previous steps is relative to the old reference: bring it to the new one.
-        // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tO + c * 32, o);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(tO + c * 32, o);
+          for (int c = 0; c < BLK; ++c)
+            if (c > row) s[c] = __float_as_uint(-CUDART_INF_F);
         }
-      }
-      m_ref = m_new;
-      if (tthread) trace(trole, 14, t);
+      };
+      load_s();
+      if (tthread) trace(trole, 11, t);
+      // Exponentials relative to the reference max m, packed to bf16, with their sum; optionally the
+      // row max of the raw logits in the same sweep.
+      // P replaces S in place: entry c/2 is written after entries c..c+3 have been read.
+      float sum, mx_raw;
+      auto sweep = [&](const float m, const bool with_max) {
+        const float neg_m = -m;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
 #pragma unroll
-      for (int c = 0; c < BLK / 64; ++c) tmem_st32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p[c * 32]));
+        for (int c = 0; c < BLK; c += 4) {
+          float x0, x1, x2, x3;
+          fma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), scale, neg_m);
+          fma2(x2, x3, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]), scale, neg_m);
+          if (with_max) {
+            mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+            mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+          }
+          x0 = ex2_approx(x0);
+          x1 = ex2_approx(x1);
+          x2 = ex2_approx(x2);
+          x3 = ex2_approx(x3);
+          add2(sum0, sum1, x0, x1);
+          add2(sum2, sum3, x2, x3);
+          s[c / 2] = cvt_bf16x2(x0, x1);
+          s[c / 2 + 1] = cvt_bf16x2(x2, x3);
+        }
+        sum = (sum0 + sum1) + (sum2 + sum3);
+        if (with_max) mx_raw = fmaxf(mx0, mx1);
+      };
+
+      // The reference max only moves when the row max has grown by more than 2^8, which is rare
+      // after the first key-block: take the exponentials against the current reference while
+      // finding the row max, and redo them (and rescale O) only if some row of the warp must move.
+      bool redo = t == 0;
+      if (!redo) {
+        sweep(m_ref, true);
+        redo = __any_sync(0xffffffffu, mx_raw * scale > m_ref + 8.f);
+      } else {
+        float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[1]));
+        float mx1 = fmaxf(__uint_as_float(s[2]), __uint_as_float(s[3]));
+        float mx2 = fmaxf(__uint_as_float(s[4]), __uint_as_float(s[5]));
+        float mx3 = fmaxf(__uint_as_float(s[6]), __uint_as_float(s[7]));
+#pragma unroll
+        for (int c = 8; c < BLK; c += 8) {
+          mx0 = max3(mx0, __uint_as_float(s[c + 0]), __uint_as_float(s[c + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+        }
+        mx_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      }
+      if (tthread) trace(trole, 12, t);
+      if (redo) {
+        const float mx = mx_raw * scale;
+        const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+        const float alpha = ex2_approx(m_ref - m_new);
+        if (t > 0) load_s();       // the first sweep recycled the registers S was in; S is still in TMEM
+        sweep(m_new, false);
+        l *= alpha;
+        if (t > 0) {
+          // O of the previous steps is relative to the old reference: bring it to the new one.
+          // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tO + c * 32, o);
+          }
+        }
+        m_ref = m_new;
+      }
+      if (tthread) trace(trole, 13, t);
+#pragma unroll
+      for (int c = 0; c < BLK / 64; ++c) tmem_st32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
       if (tthread) trace(trole, 15, t);
+      // off the critical path: running sum and the tile statistic
+      l += sum;
+      if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(sum);
     }
     if (ok) ok = mbar_wait(bar(BAR_O_DONE + x), 0, ab, 32 + x);
     float lse2 = 0.f;

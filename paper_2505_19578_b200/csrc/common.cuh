@@ -35,7 +35,7 @@ struct AttnArgs {
   float* lse;              // [n_heads, N] or null
   float* tile_stats;       // scratch: per (slot, row-block) B floats per causal tile (tensor-core path)
   int* status;             // device int[2]: {code, where}
-  long long* trace;        // optional phase trace of CTA (0,0): 4 roles x trace_cap x {tag, clock}
+  long long* trace;        // optional phase trace of CTA (0,0): 5 roles x trace_cap x {tag, clock}
   int trace_cap;
   float scale_log2;        // log2(e) / sqrt(d)
 };

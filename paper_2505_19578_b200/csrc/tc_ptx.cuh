@@ -43,18 +43,25 @@ struct Abort {
 };
 
 // Bounded wait.  Returns false if the wait ran out or another role already gave up.
+// The checks are kept off the fast path: the CTA's own abort flag (shared memory) every 64
+// polls, the time limit and the global status word (a trip to L2 that would delay the wake-up
+// by hundreds of cycles if it were made often) every 4096.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
+  long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (*ab.flag) return false;
-      if (*reinterpret_cast<volatile int*>(ab.status) != 0) {   // another CTA already gave up
-        *ab.flag = 1;
-        return false;
+      if ((it & 4095u) == 0u) {
+        if (*reinterpret_cast<volatile int*>(ab.status) != 0) {   // another CTA already gave up
+          *ab.flag = 1;
+          return false;
+        }
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitCycles) break;
       }
-      if (clock64() - t0 > kWaitCycles) break;
     }
   }
   *ab.flag = 1;
