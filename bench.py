@@ -337,7 +337,9 @@ def run_ours(args):
     # dominant kernel by time
     dom = ("pivot_dense_attn", k1, k1_tf) if k1 >= k3 else ("block_sparse_attn", k3, k3_tf)
     roofline = {
-        "kernel": f"attn_tc_kernel<{cfg.head_dim},{cfg.block}> ({dom[0]})", "bound": "tensor", "achieved": dom[2],
+        "kernel": (f"attn_pair_kernel ({dom[0]})" if (cfg.head_dim, cfg.block) == (128, 128)
+                   else f"attn_tc_kernel<{cfg.head_dim},{cfg.block}> ({dom[0]})"),
+        "bound": "tensor", "achieved": dom[2],
         "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], "unit": "TFLOP/s",
         "frac": dom[2] / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
         "peak_kind": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",

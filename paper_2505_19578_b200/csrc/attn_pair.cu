@@ -160,8 +160,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_pairs = (a.Nb + 1) >> 1;
-  const int u = n_pairs - 1 - (int)blockIdx.x;      // long row-blocks first
-  const int slot = blockIdx.y;
+  const int u = n_pairs - 1 - (int)blockIdx.y;      // long row-blocks first, across all heads
+  const int slot = blockIdx.x;
   const int h = a.heads.v[slot];
   const int g = h / a.group;
   const int list = a.lists.v[slot];
@@ -590,7 +590,7 @@ cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s) {
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
   if (e != cudaSuccess) return e;
-  attn_pair_kernel<<<dim3((a.Nb + 1) / 2, a.n_heads), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
+  attn_pair_kernel<<<dim3(a.n_heads, (a.Nb + 1) / 2), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
   return cudaGetLastError();
 }
 
