@@ -212,6 +212,32 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
                     const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
                     float gamma, int block, sp_tensor* out, uint8_t* mask_out, void* stream);
 
+/*
+ * The whole layer with HOST buffers: the same steps as sp_prefill_attn (same
+ * algorithms of the paper), with the transfers pipelined around them.  K, V and
+ * the pivots' queries are copied in first; the pivots' dense attention and the
+ * mask construction run while the members' queries are still arriving; the
+ * members run in groups of four heads, each group's outputs copied back while
+ * the next group computes.  Copies use two streams owned by the context; when the
+ * call returns everything is enqueued, and `stream` is made to wait for the last
+ * copy, so synchronising `stream` is enough before reading out_host.
+ *
+ *   q_host             host bf16 [n_q_heads, seq, head_dim], contiguous
+ *   k_host, v_host     host bf16 [n_kv_heads, seq, head_dim], contiguous
+ *   out_host           host bf16, like q_host; fully overwritten
+ *   mask_out_host      host u8 [n_q_heads, Nb, Nb] or NULL (as mask_out above)
+ *   cluster_map, pivot_heads, gamma, block   as for sp_prefill_attn
+ * Host buffers should be page-locked (cudaHostAlloc / cudaHostRegister):
+ * pageable memory works but the copies then do not overlap anything.  The
+ * buffers must stay valid and unmodified until `stream` has been synchronised.
+ * The context keeps device copies of q, k, v and out (2 q + 2 k sizes, allocated
+ * on first use, grown on demand) next to its workspace.
+ */
+int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                         int n_q_heads, int n_kv_heads, int64_t seq, int head_dim,
+                         const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
+                         float gamma, int block, void* out_host, uint8_t* mask_out_host, void* stream);
+
 /* Which attention kernel the context launches: 0 = tensor-core kernels
  * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V

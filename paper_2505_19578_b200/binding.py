@@ -29,7 +29,7 @@ EXPORTS = (
     "sp_ctx_create", "sp_ctx_destroy", "sp_workspace_bytes", "sp_ctx_reserve", "sp_get_status",
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
-    "sp_ctx_set_trace",
+    "sp_ctx_set_trace", "sp_prefill_attn_host",
 )
 
 
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
     lib.sp_block_mask_from_importance.argtypes = [P, P, I, I, F, P, P, P, P]
     lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
     lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
+    lib.sp_prefill_attn_host.argtypes = [P, P, P, P, I, I, ctypes.c_int64, I, IP, IP, I, F, I, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
@@ -182,11 +183,31 @@ class Context:
                                               _view(out), _stream(stream)),
                "sp_block_sparse_attn")
 
+    def sp_prefill_attn_host(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
+        """Host tensors (bf16, contiguous, preferably pinned): q, out [Hq, N, d]; k, v [Hkv, N, d]; mask_out u8 [Hq, Nb, Nb]."""
+        cluster_map, pivot_heads = list(cluster_map), list(pivot_heads)
+        Hq, N, d = q.shape[-3:]
+        Hkv = k.shape[-3]
+        if tuple(k.shape[-3:]) != (Hkv, N, d) or v.shape != k.shape or out.shape != q.shape:
+            raise ValueError("sp_prefill_attn_host: shapes of q, k, v, out do not match")
+        bf = torch.bfloat16
+        mp = _host_ptr(mask_out, torch.uint8, "mask_out") if mask_out is not None else None
+        _check(self._lib.sp_prefill_attn_host(self._h, _host_ptr(q, bf, "q"), _host_ptr(k, bf, "k"), _host_ptr(v, bf, "v"),
+                                              Hq, Hkv, N, d, _i32(cluster_map), _i32(pivot_heads), len(pivot_heads),
+                                              gamma, block, _host_ptr(out, bf, "out"), mp, _stream(stream)),
+               "sp_prefill_attn_host")
+
     def sp_prefill_attn(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
         cluster_map, pivot_heads = list(cluster_map), list(pivot_heads)
         _check(self._lib.sp_prefill_attn(self._h, _view(q), _view(k), _view(v), _i32(cluster_map), _i32(pivot_heads),
                                          len(pivot_heads), gamma, block, _view(out), _ptr(mask_out), _stream(stream)),
                "sp_prefill_attn")
+
+
+def _host_ptr(t, dtype, what):
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{what}: expected a contiguous host tensor of {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
 
 
 def sp_dense_pivot_attn_fixed_scratch(q, k, v, heads, block, out, importance_out=None, lse_out=None, stream=None,

@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -18,6 +19,11 @@ struct sp_ctx {
   int64_t launches = 0;
   long long* trace = nullptr;  // caller's device buffer for the phase trace, or null
   int trace_cap = 0;
+  // sp_prefill_attn_host: device copies of q, k, v, out (+ masks) and the copy streams
+  void* stage = nullptr;
+  size_t stage_bytes = 0;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  std::vector<cudaEvent_t> events;
 };
 
 namespace {
@@ -200,6 +206,10 @@ int sp_ctx_destroy(sp_ctx* ctx) {
   DeviceGuard g(ctx->device);
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->status) cudaFree(ctx->status);
+  if (ctx->stage) cudaFree(ctx->stage);
+  if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
+  if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
+  for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   delete ctx;
   return SP_OK;
 }
@@ -411,6 +421,172 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
     if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     ctx->launches += 1;
   }
+  return SP_OK;
+}
+
+int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, int n_q_heads,
+                         int n_kv_heads, int64_t seq, int head_dim, const int32_t* cluster_map,
+                         const int32_t* pivot_heads, int n_pivots, float gamma, int block, void* out_host,
+                         uint8_t* mask_out_host, void* stream) {
+  if (!ctx || !q_host || !k_host || !v_host || !out_host || !cluster_map || n_pivots < 0 || (n_pivots > 0 && !pivot_heads))
+    return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f) || n_q_heads <= 0 || n_kv_heads <= 0 || seq <= 0) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+
+  // device copies: q | k | v | out | masks, each 256-byte aligned
+  const size_t head_bytes = (size_t)seq * head_dim * sizeof(__nv_bfloat16);
+  const size_t q_bytes = align_up((size_t)n_q_heads * head_bytes), kv_bytes = align_up((size_t)n_kv_heads * head_bytes);
+  const int64_t nb = block > 0 ? seq / block : 0;
+  const size_t mask_bytes = mask_out_host ? align_up((size_t)n_q_heads * nb * nb) : 0;
+  const size_t need = 2 * q_bytes + 2 * kv_bytes + mask_bytes;
+  sp_tensor q, k, v, o;
+  auto view = [&](sp_tensor* t, void* data, int heads) {
+    t->data = data;
+    t->shape[0] = 1; t->shape[1] = heads; t->shape[2] = seq; t->shape[3] = head_dim;
+    t->stride[0] = 0; t->stride[1] = seq * head_dim; t->stride[2] = head_dim; t->stride[3] = 1;
+  };
+  // validate sizes before anything is allocated (data pointers are placeholders here)
+  view(&q, ctx, n_q_heads); view(&k, ctx, n_kv_heads); view(&v, ctx, n_kv_heads); view(&o, ctx, n_q_heads);
+  {
+    sp_tensor qa = q, ka = k, va = v, oa = o;
+    qa.data = ka.data = va.data = oa.data = reinterpret_cast<void*>(uintptr_t(256));
+    Problem chk;
+    int rc = check_problem(&qa, &ka, &va, &oa, block, &chk);
+    if (rc) return rc;
+  }
+  if (n_pivots > n_q_heads) return SP_ERR_INVALID_ARG;
+  int pivot_slot_of_head[kMaxHeads];
+  for (int h = 0; h < n_q_heads; ++h) pivot_slot_of_head[h] = -1;
+  for (int t = 0; t < n_pivots; ++t) {
+    const int h = pivot_heads[t];
+    if (h < 0 || h >= n_q_heads || pivot_slot_of_head[h] >= 0) return SP_ERR_INVALID_ARG;
+    pivot_slot_of_head[h] = t;
+  }
+  auto cluster_pivot = [&](int c) {
+    if (c < 0) return -1;
+    for (int t = 0; t < n_pivots; ++t)
+      if (cluster_map[pivot_heads[t]] == c) return t;
+    return -1;
+  };
+
+  if (need > ctx->stage_bytes) {
+    if (ctx->stage) {
+      if (cudaDeviceSynchronize() != cudaSuccess) return SP_ERR_CUDA;
+      cudaFree(ctx->stage);
+      ctx->stage = nullptr;
+      ctx->stage_bytes = 0;
+    }
+    if (cudaMalloc(&ctx->stage, need) != cudaSuccess) { cudaGetLastError(); return SP_ERR_WORKSPACE; }
+    ctx->stage_bytes = need;
+  }
+  if (!ctx->s_in && cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking) != cudaSuccess) return SP_ERR_CUDA;
+  if (!ctx->s_out && cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking) != cudaSuccess) return SP_ERR_CUDA;
+  size_t next_event = 0;
+  auto event = [&]() -> cudaEvent_t {
+    if (next_event == ctx->events.size()) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      ctx->events.push_back(e);
+    }
+    return ctx->events[next_event++];
+  };
+  // record on `from`, make `to` wait
+  auto hand_over = [&](cudaStream_t from, cudaStream_t to) {
+    cudaEvent_t e = event();
+    return e && cudaEventRecord(e, from) == cudaSuccess && cudaStreamWaitEvent(to, e, 0) == cudaSuccess;
+  };
+
+  char* base = static_cast<char*>(ctx->stage);
+  char* dq = base; char* dk = dq + q_bytes; char* dv = dk + kv_bytes; char* dout = dv + kv_bytes;
+  uint8_t* dmask = mask_out_host ? reinterpret_cast<uint8_t*>(dout + q_bytes) : nullptr;
+  view(&q, dq, n_q_heads); view(&k, dk, n_kv_heads); view(&v, dv, n_kv_heads); view(&o, dout, n_q_heads);
+  Problem p;
+  int rc = check_problem(&q, &k, &v, &o, block, &p);
+  if (rc) return rc;
+  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots);
+  if ((rc = reserve(ctx, w.total))) return rc;
+  char* ws = static_cast<char*>(ctx->ws);
+  float* imp = reinterpret_cast<float*>(ws + w.imp);
+  uint8_t* pmask = reinterpret_cast<uint8_t*>(ws + w.mask);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + w.counts);
+  int32_t* indices = reinterpret_cast<int32_t*>(ws + w.indices);
+  float* stats = reinterpret_cast<float*>(ws + w.stats);
+
+  cudaStream_t sc = static_cast<cudaStream_t>(stream), sin = ctx->s_in, sout = ctx->s_out;
+  const char* hq = static_cast<const char*>(q_host);
+  char* ho = static_cast<char*>(out_host);
+  auto copy_in_head = [&](int h) {
+    return cudaMemcpyAsync(dq + (size_t)h * head_bytes, hq + (size_t)h * head_bytes, head_bytes, cudaMemcpyHostToDevice, sin) == cudaSuccess;
+  };
+  auto copy_out_head = [&](int h) {
+    return cudaMemcpyAsync(ho + (size_t)h * head_bytes, dout + (size_t)h * head_bytes, head_bytes, cudaMemcpyDeviceToHost, sout) == cudaSuccess;
+  };
+
+  // The copy streams start after whatever the caller's stream already holds (an earlier call on
+  // this context may still be reading the device copies).
+  if (!hand_over(sc, sin) || !hand_over(sc, sout)) return SP_ERR_CUDA;
+
+  // in: K, V, the pivots' queries; compute: step 1 + step 2 while the members' queries arrive
+  if (cudaMemcpyAsync(dk, k_host, (size_t)n_kv_heads * head_bytes, cudaMemcpyHostToDevice, sin) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v_host, (size_t)n_kv_heads * head_bytes, cudaMemcpyHostToDevice, sin) != cudaSuccess)
+    return SP_ERR_CUDA;
+  for (int t = 0; t < n_pivots; ++t)
+    if (!copy_in_head(pivot_heads[t])) return SP_ERR_CUDA;
+  if (!hand_over(sin, sc)) return SP_ERR_CUDA;
+
+  AttnArgs a = base_args(ctx, p, &q, &k, &v, &o);
+  a.n_heads = n_pivots;
+  for (int t = 0; t < n_pivots; ++t) { a.heads.v[t] = pivot_heads[t]; a.lists.v[t] = -1; }
+  a.importance = imp;
+  a.tile_stats = stats;
+  if ((rc = launch_attn(ctx, a, sc))) return rc;
+  if (n_pivots > 0) {
+    MaskArgs m{imp, n_pivots, p.Nb, (double)gamma, pmask, counts, indices};
+    if (launch_block_mask(m, sc) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+    if (!hand_over(sc, sout)) return SP_ERR_CUDA;
+    for (int t = 0; t < n_pivots; ++t)
+      if (!copy_out_head(pivot_heads[t])) return SP_ERR_CUDA;
+  }
+
+  // members in groups: queries in, block-sparse attention, outputs out, each on its own stream
+  HeadTable mask_src;
+  int members[kMaxHeads], member_list[kMaxHeads], n_members = 0;
+  for (int h = 0; h < p.Hq; ++h) {
+    if (pivot_slot_of_head[h] >= 0) { mask_src.v[h] = pivot_slot_of_head[h]; continue; }
+    const int t = cluster_pivot(cluster_map[h]);
+    mask_src.v[h] = t;
+    members[n_members] = h;
+    member_list[n_members] = t;
+    ++n_members;
+  }
+  constexpr int kGroup = 4;
+  for (int g0 = 0; g0 < n_members; g0 += kGroup) {
+    const int g1 = g0 + kGroup < n_members ? g0 + kGroup : n_members;
+    for (int x = g0; x < g1; ++x)
+      if (!copy_in_head(members[x])) return SP_ERR_CUDA;
+    if (!hand_over(sin, sc)) return SP_ERR_CUDA;
+    AttnArgs b = base_args(ctx, p, &q, &k, &v, &o);
+    b.counts = counts;
+    b.indices = indices;
+    b.n_heads = g1 - g0;
+    for (int x = g0; x < g1; ++x) { b.heads.v[x - g0] = members[x]; b.lists.v[x - g0] = member_list[x]; }
+    if ((rc = launch_attn(ctx, b, sc))) return rc;
+    if (!hand_over(sc, sout)) return SP_ERR_CUDA;
+    for (int x = g0; x < g1; ++x)
+      if (!copy_out_head(members[x])) return SP_ERR_CUDA;
+  }
+  if (mask_out_host) {
+    gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, sc>>>(pmask, mask_src, p.Nb, dmask);
+    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+    if (!hand_over(sc, sout)) return SP_ERR_CUDA;
+    if (cudaMemcpyAsync(mask_out_host, dmask, (size_t)p.Hq * p.Nb * p.Nb, cudaMemcpyDeviceToHost, sout) != cudaSuccess)
+      return SP_ERR_CUDA;
+  }
+  // the caller's stream ends after the last copy out (and after the last copy in)
+  if (!hand_over(sout, sc) || !hand_over(sin, sc)) return SP_ERR_CUDA;
   return SP_OK;
 }
 

@@ -218,6 +218,33 @@ def test_prefill_degenerate_head_sets(binding, kernel):
     _check_layer(L, 1.5, out, mask)
 
 
+@pytest.mark.parametrize("name,seq", [("llama8b_32k", 4096), ("tiny", 1024), ("qwen7b_64k", 2048)])
+def test_prefill_host_buffers_equal_device_call(binding, name, seq):
+    # same kernels on the same bits, only the transfers are pipelined around them: outputs must be identical
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=4)
+    cfg = L["cfg"]
+    Nb = cfg.seq // cfg.block
+    out_d, mask_d = _run_layer(binding, L, 0.9, "tc")
+    _check_layer(L, 0.9, out_d, mask_d)
+    ctx = binding.Context()
+    hq, hk, hv = (L[x].contiguous().pin_memory() for x in ("q", "k", "v"))
+    for rep in range(2):                                       # second call reuses the device copies
+        hout = torch.full(hq.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+        hmask = torch.full((cfg.n_q_heads, Nb, Nb), 9, dtype=torch.uint8).pin_memory()
+        ctx.sp_prefill_attn_host(hq, hk, hv, L["cluster_map"], L["pivot_heads"], 0.9, cfg.block, hout,
+                                 mask_out=hmask if rep == 0 else None)
+        _sync_ok(ctx)
+        assert torch.equal(hout.view(torch.int16), out_d.cpu().view(torch.int16))
+        if rep == 0:
+            assert torch.equal(hmask, mask_d.cpu())
+    # pageable host memory is accepted too
+    pout = torch.empty(hq.shape, dtype=torch.bfloat16)
+    ctx.sp_prefill_attn_host(L["q"].contiguous(), L["k"].contiguous(), L["v"].contiguous(), L["cluster_map"],
+                             L["pivot_heads"], 0.9, cfg.block, pout)
+    _sync_ok(ctx)
+    assert torch.equal(pout.view(torch.int16), out_d.cpu().view(torch.int16))
+
+
 def test_tc_and_simt_kernels_agree_on_importance(binding):
     # two different algorithms for the tile mass (one pass + spilled statistics vs two passes)
     q, k, v = _rand_layer(7, 2, 1, 1024, 128, scale=3.0)
