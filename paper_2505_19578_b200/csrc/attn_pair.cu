@@ -14,14 +14,13 @@
 // that tile alone.  (Dense: the union is 0..2u+1, the last key-block is B's
 // diagonal tile only.)
 //
-// Warp roles (384 threads):
+// Warp roles (320 threads):
 //   warps 0-3   softmax of tile A: thread t owns query row t = TMEM lane t
 //   warps 4-7   softmax of tile B
 //   warp  8     MMA issuer, owner of the TMEM allocation (all 512 columns:
 //               S_A, S_B, O_A, O_B, 128 fp32 columns each)
 //   warp  9     producer: merges the two lists, TMA loads of Q (once) and of
 //               the K and V tiles into two-stage rings (128-byte swizzle)
-//   warps 10-11 idle (they only give their registers to the softmax warps)
 //
 // Order of the MMAs, per merged key-block n:  PV_A(n), QK_A(n+1), PV_B(n),
 // QK_B(n+1), all issued by one thread: while the softmax warps of A work on
@@ -49,7 +48,7 @@ using namespace tc;
 
 constexpr int D = 128;      // head_dim
 constexpr int BLK = 128;    // block
-constexpr int kThreadsPair = 384;
+constexpr int kThreadsPair = 320;
 constexpr int kStages = 2;  // K ring and V ring depth
 
 // shared-memory plan (bytes)
@@ -106,6 +105,26 @@ __device__ __forceinline__ void reg_fence32(uint32_t* r) {
                  "+r"(r[30]), "+r"(r[31])::"memory");
 }
 
+// 16 consecutive 32-bit columns of this thread's TMEM lane <-> registers
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -132,11 +151,6 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
 }
-
-template <int N>
-__device__ __forceinline__ void set_regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N>
-__device__ __forceinline__ void set_regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // One tile's geometry as seen by every role.
 struct TileInfo {
@@ -217,7 +231,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   const uint32_t tmem = *tmem_slot;
 
   if (warp >= 8) {
-    set_regs_dec<112>();
     if (warp == 9) {
       // ---------------------------------------------------------- producer
       if (any_work) {
@@ -383,7 +396,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue of tile x
-    set_regs_inc<192>();
     const int x = warp >> 2;
     const int row = threadIdx.x & 127;                 // TMEM lane == query row inside the tile
     const int i = x ? tile[1].i : tile[0].i, cnt = x ? tile[1].cnt : tile[0].cnt;
@@ -406,104 +418,103 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       if (!ok) break;
       tc_fence_after();
       if (tthread) trace(trole, 10, t);
-      uint32_t s[BLK];
-      auto load_s = [&]() {
+      // The 128 columns are taken as four chunks of 32, each an online-softmax step of its own:
+      // chunk max, (rarely) a move of the reference, exponentials, P chunk back into the columns
+      // that earlier chunks have already given up.  The next chunk's load is in flight meanwhile.
+      const bool diag = j == i;
+      float tile_sum = 0.f;
+      uint32_t sa[32], sb[32];
+      tmem_ld32_async(tS, sa);
+      auto chunk = [&](uint32_t* sc, const int c) {     // c: chunk index 0..3 (columns 32c .. 32c+31)
+        if (diag) {
 #pragma unroll
-        for (int c = 0; c < BLK / 32; ++c) tmem_ld32_async(tS + c * 32, &s[c * 32]);
-        tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < BLK / 32; ++c) reg_fence32(&s[c * 32]);
-        if (j == i) {
-#pragma unroll
-          for (int c = 0; c < BLK; ++c)
-            if (c > row) s[c] = __float_as_uint(-CUDART_INF_F);
+          for (int e = 0; e < 32; ++e)
+            if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
         }
-      };
-      load_s();
-      if (tthread) trace(trole, 11, t);
-      // Exponentials relative to the reference max m, packed to bf16, with their sum; optionally the
-      // row max of the raw logits in the same sweep.
-      // P replaces S in place: entry c/2 is written after entries c..c+3 have been read.
-      float sum, mx_raw;
-      auto sweep = [&](const float m, const bool with_max) {
-        const float neg_m = -m;
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-        float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+        float mx0 = max3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
+        float mx1 = max3(__uint_as_float(sc[3]), __uint_as_float(sc[4]), __uint_as_float(sc[5]));
+        float mx2 = max3(__uint_as_float(sc[6]), __uint_as_float(sc[7]), __uint_as_float(sc[8]));
+        float mx3 = max3(__uint_as_float(sc[9]), __uint_as_float(sc[10]), __uint_as_float(sc[11]));
 #pragma unroll
-        for (int c = 0; c < BLK; c += 4) {
-          float x0, x1, x2, x3;
-          fma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), scale, neg_m);
-          fma2(x2, x3, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]), scale, neg_m);
-          if (with_max) {
-            mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-            mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+        for (int e = 12; e < 28; e += 8) {
+          mx0 = max3(mx0, __uint_as_float(sc[e + 0]), __uint_as_float(sc[e + 1]));
+          mx1 = max3(mx1, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]));
+          mx2 = max3(mx2, __uint_as_float(sc[e + 4]), __uint_as_float(sc[e + 5]));
+          mx3 = max3(mx3, __uint_as_float(sc[e + 6]), __uint_as_float(sc[e + 7]));
+        }
+        mx0 = max3(mx0, __uint_as_float(sc[28]), __uint_as_float(sc[29]));
+        mx1 = max3(mx1, __uint_as_float(sc[30]), __uint_as_float(sc[31]));
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
+        // the reference max only moves when the row max has grown by more than 2^8 (rare after the
+        // first chunk of the first key-block; a fully masked chunk has mx = -inf and leaves it alone)
+        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+          const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+          const float alpha = ex2_approx(m_ref - m_new);
+          if (t > 0) {
+            // O of the previous steps is relative to the old reference: bring it to the new one.
+            // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+#pragma unroll 1
+            for (int oc = 0; oc < D / 32; ++oc) {
+              uint32_t o[32];
+              tmem_ld32(tO + oc * 32, o);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+              tmem_st32(tO + oc * 32, o);
+            }
           }
+          // the P chunks of this key-block that are already stored
+#pragma unroll 1
+          for (int pc = 0; pc < c; ++pc) {
+            uint32_t pp[16];
+            tmem_ld16(tS + pc * 16, pp);
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+              pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
+            tmem_st16(tS + pc * 16, pp);
+          }
+          l *= alpha;
+          tile_sum *= alpha;
+          m_ref = m_new;
+        }
+        const float neg_m = -m_ref;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          float x0, x1, x2, x3;
+          fma2(x0, x1, __uint_as_float(sc[e]), __uint_as_float(sc[e + 1]), scale, neg_m);
+          fma2(x2, x3, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]), scale, neg_m);
           x0 = ex2_approx(x0);
           x1 = ex2_approx(x1);
           x2 = ex2_approx(x2);
           x3 = ex2_approx(x3);
           add2(sum0, sum1, x0, x1);
           add2(sum2, sum3, x2, x3);
-          s[c / 2] = cvt_bf16x2(x0, x1);
-          s[c / 2 + 1] = cvt_bf16x2(x2, x3);
+          pk[e / 2] = cvt_bf16x2(x0, x1);
+          pk[e / 2 + 1] = cvt_bf16x2(x2, x3);
         }
-        sum = (sum0 + sum1) + (sum2 + sum3);
-        if (with_max) mx_raw = fmaxf(mx0, mx1);
+        tile_sum += (sum0 + sum1) + (sum2 + sum3);
+        tmem_st16(tS + c * 16, pk);
       };
-
-      // The reference max only moves when the row max has grown by more than 2^8, which is rare
-      // after the first key-block: take the exponentials against the current reference while
-      // finding the row max, and redo them (and rescale O) only if some row of the warp must move.
-      bool redo = t == 0;
-      if (!redo) {
-        sweep(m_ref, true);
-        redo = __any_sync(0xffffffffu, mx_raw * scale > m_ref + 8.f);
-      } else {
-        float mx0 = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[1]));
-        float mx1 = fmaxf(__uint_as_float(s[2]), __uint_as_float(s[3]));
-        float mx2 = fmaxf(__uint_as_float(s[4]), __uint_as_float(s[5]));
-        float mx3 = fmaxf(__uint_as_float(s[6]), __uint_as_float(s[7]));
-#pragma unroll
-        for (int c = 8; c < BLK; c += 8) {
-          mx0 = max3(mx0, __uint_as_float(s[c + 0]), __uint_as_float(s[c + 1]));
-          mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-          mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-          mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-        }
-        mx_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      }
-      if (tthread) trace(trole, 12, t);
-      if (redo) {
-        const float mx = mx_raw * scale;
-        const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
-        const float alpha = ex2_approx(m_ref - m_new);
-        if (t > 0) load_s();       // the first sweep recycled the registers S was in; S is still in TMEM
-        sweep(m_new, false);
-        l *= alpha;
-        if (t > 0) {
-          // O of the previous steps is relative to the old reference: bring it to the new one.
-          // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tO + c * 32, o);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tO + c * 32, o);
-          }
-        }
-        m_ref = m_new;
+#pragma unroll 1
+      for (int c = 0; c < 4; c += 2) {
+        tmem_ld_wait();
+        reg_fence32(sa);
+        tmem_ld32_async(tS + (c + 1) * 32, sb);
+        chunk(sa, c);
+        tmem_ld_wait();
+        reg_fence32(sb);
+        if (c == 0) tmem_ld32_async(tS + 64, sa);
+        chunk(sb, c + 1);
       }
       if (tthread) trace(trole, 13, t);
-#pragma unroll
-      for (int c = 0; c < BLK / 64; ++c) tmem_st32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
       if (tthread) trace(trole, 15, t);
       // off the critical path: running sum and the tile statistic
-      l += sum;
-      if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(sum);
+      l += tile_sum;
+      if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(tile_sum);
     }
     if (ok) ok = mbar_wait(bar(BAR_O_DONE + x), 0, ab, 32 + x);
     float lse2 = 0.f;
@@ -511,7 +522,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       tc_fence_after();
       const float inv_l = 1.f / l;
       __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
         uint32_t o[32];
         tmem_ld32(tO + c * 32, o);
