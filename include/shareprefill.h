@@ -238,6 +238,50 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
                          const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
                          float gamma, int block, void* out_host, uint8_t* mask_out_host, void* stream);
 
+/*
+ * Paper-literal pattern construction (the library's default pattern is the true
+ * softmax mass per block, cut per row-block; these three calls follow the text
+ * of the paper instead, so that the two can be compared).
+ *
+ * sp_pooled_logits - the block-wise average of the QK values, A~ (Section 5.2,
+ *   "Sparse Attention Computation": computed next to the output; a block that is
+ *   not computed gets -infinity).  Entry [t][i][j], j <= i, is the mean of
+ *   q_r . k_c / sqrt(head_dim) over the visible (c <= r) entries of the block of
+ *   head heads[t]; entries with j > i are -infinity.  The mean over a full block
+ *   equals the product of the block means of Q and K, which is how it is
+ *   computed (fp32).
+ *     heads host [n_heads]; pooled_out device fp32 [n_heads, Nb, Nb].
+ *
+ * sp_pattern_from_pooled - Algorithm "Construct Pivotal Pattern": softmax of the
+ *   block averages along each row-block, the last row kept as the pivotal
+ *   representative a~, the map flattened and normalised by its total, sorted
+ *   descending (equal scores: smaller row-major index first), minimum budget K
+ *   whose scores sum to >= gamma (every existing block if they never do), index
+ *   set -> mask.  A row-block left without a selected block receives its diagonal
+ *   block.  Outputs as for sp_block_mask_from_importance (mask_out required),
+ *   plus last_row_out device fp32 [n_maps, nb] or NULL.
+ *
+ * sp_determine_pattern - Algorithm "Determine Sparse Pattern": a^ = softmax of
+ *   the pooled QK values of the last block of queries against every key-block,
+ *   d_sparse = sqrt(JSD(a^ || uniform)), d_sim = sqrt(JSD(a^ || a~)) (natural
+ *   logarithm), pattern = shared pivot iff d_sparse < delta and d_sim < tau,
+ *   else vertical-slash.
+ *     pivot_last_rows device fp32 [n_rows, Nb] (a~ of the pivots, as written by
+ *     sp_pattern_from_pooled); row_of_head host [n_heads]: which row each head is
+ *     compared with, -1 = none (d_sim = +infinity).
+ *     pattern_out device i32 [n_heads]: 0 = shared pivot, 1 = vertical-slash;
+ *     dist_out device fp32 [n_heads, 2] = (d_sparse, d_sim), or NULL.
+ */
+int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads,
+                     int n_heads, int block, float* pooled_out, void* stream);
+int sp_pattern_from_pooled(sp_ctx* ctx, const float* pooled, int n_maps, int nb, float gamma,
+                           uint8_t* mask_out, int32_t* counts_out, int32_t* indices_out,
+                           float* last_row_out, void* stream);
+int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads,
+                         int n_heads, int block, const float* pivot_last_rows,
+                         const int32_t* row_of_head, float delta, float tau, int32_t* pattern_out,
+                         float* dist_out, void* stream);
+
 /* Which attention kernel the context launches: 0 = tensor-core kernels
  * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V

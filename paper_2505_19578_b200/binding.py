@@ -29,7 +29,8 @@ EXPORTS = (
     "sp_ctx_create", "sp_ctx_destroy", "sp_workspace_bytes", "sp_ctx_reserve", "sp_get_status",
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
-    "sp_ctx_set_trace", "sp_prefill_attn_host",
+    "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
+    "sp_determine_pattern",
 )
 
 
@@ -72,6 +73,9 @@ def load() -> ctypes.CDLL:
     lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
     lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
     lib.sp_prefill_attn_host.argtypes = [P, P, P, P, I, I, ctypes.c_int64, I, IP, IP, I, F, I, P, P, P]
+    lib.sp_pooled_logits.argtypes = [P, T, T, IP, I, I, P, P]
+    lib.sp_pattern_from_pooled.argtypes = [P, P, I, I, F, P, P, P, P, P]
+    lib.sp_determine_pattern.argtypes = [P, T, T, IP, I, I, P, IP, F, F, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
@@ -182,6 +186,28 @@ class Context:
                                               _i32(list_of_head), _ptr(counts), _ptr(indices), n_lists, block,
                                               _view(out), _stream(stream)),
                "sp_block_sparse_attn")
+
+    # ---- paper-literal pattern construction and decision -------------------
+
+    def sp_pooled_logits(self, q, k, heads, block, pooled_out, stream=None):
+        heads = list(heads)
+        _check(self._lib.sp_pooled_logits(self._h, _view(q), _view(k), _i32(heads), len(heads), block, _ptr(pooled_out),
+                                          _stream(stream)), "sp_pooled_logits")
+
+    def sp_pattern_from_pooled(self, pooled, gamma, mask_out, counts_out, indices_out, last_row_out=None, stream=None):
+        n_maps, nb, nb2 = pooled.shape
+        assert nb == nb2 and pooled.dtype == torch.float32 and pooled.is_contiguous()
+        _check(self._lib.sp_pattern_from_pooled(self._h, _ptr(pooled), n_maps, nb, gamma, _ptr(mask_out), _ptr(counts_out),
+                                                _ptr(indices_out), _ptr(last_row_out), _stream(stream)),
+               "sp_pattern_from_pooled")
+
+    def sp_determine_pattern(self, q, k, heads, block, pivot_last_rows, row_of_head, delta, tau, pattern_out,
+                             dist_out=None, stream=None):
+        heads, row_of_head = list(heads), list(row_of_head)
+        assert len(heads) == len(row_of_head)
+        _check(self._lib.sp_determine_pattern(self._h, _view(q), _view(k), _i32(heads), len(heads), block,
+                                              _ptr(pivot_last_rows), _i32(row_of_head), delta, tau, _ptr(pattern_out),
+                                              _ptr(dist_out), _stream(stream)), "sp_determine_pattern")
 
     def sp_prefill_attn_host(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
         """Host tensors (bf16, contiguous, preferably pinned): q, out [Hq, N, d]; k, v [Hkv, N, d]; mask_out u8 [Hq, Nb, Nb]."""

@@ -590,4 +590,87 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
   return SP_OK;
 }
 
+namespace {
+// q, k views -> PooledArgs (problem checked by the caller)
+PooledArgs pooled_args(const Problem& p, const sp_tensor* q, const sp_tensor* k, const int32_t* heads, int n_heads) {
+  PooledArgs a;
+  memset(&a, 0, sizeof(a));
+  a.q = static_cast<const __nv_bfloat16*>(q->data);
+  a.k = static_cast<const __nv_bfloat16*>(k->data);
+  a.q_sh = q->stride[1]; a.q_sn = q->stride[2];
+  a.k_sh = k->stride[1]; a.k_sn = k->stride[2];
+  a.group = p.Hq / p.Hkv; a.B = p.B; a.Nb = p.Nb; a.d = p.d; a.n_heads = n_heads;
+  for (int t = 0; t < n_heads; ++t) a.heads.v[t] = heads[t];
+  a.scale = (float)(1.0 / sqrt((double)p.d));
+  return a;
+}
+}  // namespace
+
+int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads, int n_heads, int block,
+                     float* pooled_out, void* stream) {
+  if (!ctx || !heads || n_heads < 0 || !pooled_out) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, k, q, block, &p);
+  if (rc) return rc;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  for (int t = 0; t < n_heads; ++t)
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  if ((rc = reserve(ctx, align_up(pooled_scratch_floats(n_heads, p.Nb, p.d) * sizeof(float))))) return rc;
+  PooledArgs a = pooled_args(p, q, k, heads, n_heads);
+  a.qbar = static_cast<float*>(ctx->ws);
+  a.kbar = a.qbar + (size_t)n_heads * p.Nb * p.d;
+  a.diag = a.kbar + (size_t)n_heads * p.Nb * p.d;
+  a.pooled = pooled_out;
+  if (launch_pooled_logits(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  ctx->launches += 2;
+  return SP_OK;
+}
+
+int sp_pattern_from_pooled(sp_ctx* ctx, const float* pooled, int n_maps, int nb, float gamma, uint8_t* mask_out,
+                           int32_t* counts_out, int32_t* indices_out, float* last_row_out, void* stream) {
+  if (!ctx || !pooled || !mask_out || !counts_out || !indices_out || n_maps < 0 || nb <= 0) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  if (nb > kMaxNb) return SP_ERR_UNSUPPORTED;
+  if (n_maps == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  int rc = reserve(ctx, align_up((size_t)n_maps * nb * nb * sizeof(float)));
+  if (rc) return rc;
+  if (launch_pattern_from_pooled(pooled, n_maps, nb, (double)gamma, static_cast<float*>(ctx->ws), mask_out, counts_out,
+                                 indices_out, last_row_out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SP_ERR_CUDA;
+  ctx->launches += 3;
+  return SP_OK;
+}
+
+int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads, int n_heads, int block,
+                         const float* pivot_last_rows, const int32_t* row_of_head, float delta, float tau,
+                         int32_t* pattern_out, float* dist_out, void* stream) {
+  if (!ctx || !heads || n_heads < 0 || !pattern_out || !row_of_head) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, k, q, block, &p);
+  if (rc) return rc;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  HeadTable rows;
+  for (int t = 0; t < n_heads; ++t) {
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+    if (row_of_head[t] >= 0 && !pivot_last_rows) return SP_ERR_INVALID_ARG;
+    rows.v[t] = row_of_head[t] < 0 ? -1 : row_of_head[t];
+  }
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  if ((rc = reserve(ctx, align_up((size_t)n_heads * p.Nb * sizeof(float))))) return rc;
+  PooledArgs a = pooled_args(p, q, k, heads, n_heads);
+  a.pooled = static_cast<float*>(ctx->ws);
+  if (launch_determine_pattern(a, pivot_last_rows, rows, delta, tau, pattern_out, dist_out,
+                               static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SP_ERR_CUDA;
+  ctx->launches += 2;
+  return SP_OK;
+}
+
 }  // extern "C"

@@ -49,6 +49,20 @@ struct MaskArgs {
   int32_t* indices;
 };
 
+// Block-averaged QK values (paper-literal pattern construction / decision).  Strides in elements.
+struct PooledArgs {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  int64_t q_sh, q_sn, k_sh, k_sn;
+  int group, B, Nb, d, n_heads;
+  HeadTable heads;
+  float scale;     // 1 / sqrt(d)
+  float* qbar;     // scratch [n_heads, Nb, d]: block means of Q
+  float* kbar;     // scratch [n_heads, Nb, d]: block means of K (of the head's KV head)
+  float* diag;     // scratch [n_heads, Nb]: average of the diagonal block's visible entries, scaled
+  float* pooled;   // out [n_heads, Nb, Nb]  (launch_determine_pattern: [n_heads, Nb], the last row only)
+};
+
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA, one row-block per CTA
@@ -60,6 +74,13 @@ cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s)
 constexpr size_t kFixedScratchBytes = 64ull << 20;
 cudaError_t launch_block_mask(const MaskArgs& a, cudaStream_t s);
 cudaError_t launch_fill_causal_mask(uint8_t* mask, int nb, cudaStream_t s);
+size_t pooled_scratch_floats(int n_heads, int Nb, int d);
+cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s);
+cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
+                                       uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
+                                       cudaStream_t s);
+cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,
+                                     float delta, float tau, int32_t* pattern, float* dist, cudaStream_t s);
 
 // bytes of per-tile softmax statistics the tensor-core kernel spills for one head
 inline size_t tile_stats_bytes_per_head(int Nb, int B) {

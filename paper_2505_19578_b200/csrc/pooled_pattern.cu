@@ -1,0 +1,384 @@
+// Paper-literal pattern construction and decision.
+//
+//   Section 5.2, "Sparse Attention Computation": next to the output the kernel
+//   yields the block-wise average of the QK values, A~.
+//   Algorithm "Construct Pivotal Pattern": A~ = softmax(A~); a~ = its last row;
+//   flatten and normalise; sort; minimum budget K whose scores sum to gamma;
+//   index set -> mask.
+//   Algorithm "Determine Sparse Pattern": a^ = softmax(pool(Q^ K^T)/sqrt(d)) for
+//   the last block of queries, d_sparse = sqrt(JSD(a^ || u)), d_sim =
+//   sqrt(JSD(a^ || a~)); shared pivot iff d_sparse < delta and d_sim < tau.
+//
+// The average of q_r . k_c over a full block is the product of the block means
+// of Q and of K, so the map needs no pass over the tiles: block means of Q and K
+// (one read of the two tensors), one small product per block, and the diagonal
+// block (only its visible half is averaged) through a running key prefix sum.
+// The global cut is a radix select on the score bits with float64 bin sums
+// (three passes of 11 + 11 + 10 bits), followed by an ordered pass that breaks
+// ties towards the smaller flattened index.  All of it is HBM- and latency-sized
+// work (a few MB per head).
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace sp {
+namespace {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ---- block means of Q and K, and the average of the diagonal block ------------------------
+// grid (Nb, n_heads), d threads: thread = one head-dim column.
+__global__ void block_means_kernel(const PooledArgs a) {
+  __shared__ float red[4];
+  const int i = blockIdx.x, slot = blockIdx.y, col = threadIdx.x;
+  const int h = a.heads.v[slot], g = h / a.group;
+  const __nv_bfloat16* q = a.q + (size_t)h * a.q_sh + (size_t)i * a.B * a.q_sn + col;
+  const __nv_bfloat16* k = a.k + (size_t)g * a.k_sh + (size_t)i * a.B * a.k_sn + col;
+  float qsum = 0.f, kcum = 0.f, acc = 0.f;
+  for (int r = 0; r < a.B; ++r) {
+    const float qv = __bfloat162float(q[(size_t)r * a.q_sn]);
+    kcum += __bfloat162float(k[(size_t)r * a.k_sn]);
+    qsum += qv;
+    acc = fmaf(qv, kcum, acc);          // q_r . (k_0 + ... + k_r): the visible half of the diagonal block
+  }
+  const float inv = 1.f / (float)a.B;
+  a.qbar[((size_t)slot * a.Nb + i) * a.d + col] = qsum * inv;
+  a.kbar[((size_t)slot * a.Nb + i) * a.d + col] = kcum * inv;
+  acc = warp_sum(acc);
+  if ((col & 31) == 0) red[col >> 5] = acc;
+  __syncthreads();
+  if (col == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    a.diag[(size_t)slot * a.Nb + i] = t * a.scale / (0.5f * (float)a.B * (float)(a.B + 1));
+  }
+}
+
+// ---- A~[i][j] = qbar_i . kbar_j / sqrt(d)  (j < i), diagonal from above, -inf for j > i ------
+// grid (Nb, n_heads), 128 threads: warp w takes key-blocks w, w+4, ...
+__global__ void pooled_logits_kernel(const PooledArgs a) {
+  const int i = blockIdx.x, slot = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* qb = a.qbar + ((size_t)slot * a.Nb + i) * a.d;
+  float* out = a.pooled + ((size_t)slot * a.Nb + i) * a.Nb;
+  const int per = a.d / 32;              // 2 or 4 consecutive columns per lane
+  float qv[4];
+  for (int e = 0; e < per; ++e) qv[e] = qb[lane * per + e];
+  for (int j = warp; j < i; j += 4) {
+    const float* kb = a.kbar + ((size_t)slot * a.Nb + j) * a.d;
+    float acc = 0.f;
+    for (int e = 0; e < per; ++e) acc = fmaf(qv[e], kb[lane * per + e], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) out[j] = acc * a.scale;
+  }
+  if (threadIdx.x == 0) out[i] = a.diag[(size_t)slot * a.Nb + i];
+  for (int j = i + 1 + (int)threadIdx.x; j < a.Nb; j += blockDim.x) out[j] = -CUDART_INF_F;
+}
+
+// ---- row-wise softmax of the block averages; one warp per row -------------------------------
+__global__ void pooled_softmax_kernel(const float* __restrict__ pooled, int n_maps, int nb, float* __restrict__ scores,
+                                      float* __restrict__ last_row) {
+  const int lane = threadIdx.x & 31;
+  const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (w >= (long)n_maps * nb) return;
+  const int mp = (int)(w / nb), i = (int)(w % nb);
+  const float* row = pooled + ((size_t)mp * nb + i) * nb;
+  float* out = scores + ((size_t)mp * nb + i) * nb;
+  float m = -CUDART_INF_F;
+  for (int j = lane; j <= i; j += 32) m = fmaxf(m, row[j]);
+  m = warp_max(m);
+  float s = 0.f;
+  for (int j = lane; j <= i; j += 32) s += expf(row[j] - m);
+  s = warp_sum(s);
+  const float inv = 1.f / s;
+  for (int j = lane; j < nb; j += 32) {
+    const float p = j <= i ? expf(row[j] - m) * inv : 0.f;
+    out[j] = p;
+    if (last_row && i == nb - 1) last_row[(size_t)mp * nb + j] = p;
+  }
+}
+
+// ---- global cumulative cut over one map; one CTA of 1024 threads per map ---------------------
+constexpr int kSelThreads = 1024;
+constexpr int kBins = 2048;
+
+struct SelShared {
+  unsigned int count[kBins];
+  double sum[kBins];
+  double total, cum_above;
+  unsigned int prefix, k_eq, running, select_all;
+  unsigned int warp_cnt[kSelThreads / 32];
+};
+
+__global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float* __restrict__ scores, int nb, double gamma,
+                                                                    uint8_t* __restrict__ mask) {
+  extern __shared__ unsigned char sel_raw[];
+  SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
+  const int mp = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* sc = scores + (size_t)mp * nb * nb;
+  uint8_t* mk = mask + (size_t)mp * nb * nb;
+  const long n = (long)nb * nb;
+
+  // total of the map (each row sums to 1 up to rounding), float64
+  if (tid == 0) { sh.total = 0.0; sh.cum_above = 0.0; sh.prefix = 0u; sh.select_all = 0u; sh.running = 0u; }
+  __syncthreads();
+  {
+    double t = 0.0;
+    for (long e = tid; e < n; e += kSelThreads) {
+      const int i = (int)(e / nb), j = (int)(e % nb);
+      if (j <= i) t += (double)sc[e];
+    }
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) atomicAdd(&sh.total, t);
+  }
+  __syncthreads();
+  const double inv_total = 1.0 / sh.total;
+
+  // radix select, most significant digit first: digits of 11, 11, 10 bits
+  const int shift[3] = {21, 10, 0};
+  const unsigned int dmask[3] = {0x7FFu, 0x7FFu, 0x3FFu};
+  for (int pass = 0; pass < 3 && !sh.select_all; ++pass) {
+    for (int b = tid; b < kBins; b += kSelThreads) { sh.count[b] = 0u; sh.sum[b] = 0.0; }
+    __syncthreads();
+    const unsigned int prefix = sh.prefix;
+    const int above = shift[pass] + (pass == 0 ? 11 : (pass == 1 ? 11 : 10));   // bits above this digit
+    for (long e = tid; e < n; e += kSelThreads) {
+      const int i = (int)(e / nb), j = (int)(e % nb);
+      if (j > i) continue;
+      const unsigned int bits = __float_as_uint(sc[e]);
+      if (pass > 0 && (bits >> above) != prefix) continue;
+      const unsigned int dgt = (bits >> shift[pass]) & dmask[pass];
+      atomicAdd(&sh.count[dgt], 1u);
+      atomicAdd(&sh.sum[dgt], (double)sc[e] * inv_total);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      double cum = sh.cum_above;
+      int b = (int)dmask[pass];
+      bool found = false;
+      int lowest = -1;                    // lowest non-empty digit seen
+      double cum_before_lowest = cum;
+      for (; b >= 0; --b) {
+        if (sh.count[b] == 0u) continue;
+        lowest = b;
+        cum_before_lowest = cum;
+        if (cum + sh.sum[b] >= gamma) { found = true; break; }
+        cum += sh.sum[b];
+      }
+      if (!found && pass > 0 && lowest >= 0) {
+        // the digit above said the cut lies in this group; its members were summed in another order
+        // and fall short by rounding: the cut is the group's smallest value
+        found = true;
+        b = lowest;
+        cum = cum_before_lowest;
+      }
+      if (!found) {
+        sh.select_all = 1u;                       // the scores never reach gamma: every block that exists
+      } else {
+        sh.cum_above = cum;
+        sh.prefix = (prefix << (pass == 2 ? 10 : 11)) | (unsigned int)b;
+        if (pass == 2) {
+          // prefix is now the bit pattern of the cut value; how many of its copies are needed
+          const double v = (double)__uint_as_float(sh.prefix) * inv_total;
+          unsigned int k = 0;
+          double c = cum;
+          const unsigned int n_eq = sh.count[b];
+          do { c += v; ++k; } while (c < gamma && k < n_eq);
+          sh.k_eq = k;
+        }
+      }
+    }
+    __syncthreads();
+  }
+
+  // ordered marking: everything above the cut value, and the first k_eq copies of it in row-major order
+  const bool all = sh.select_all != 0u;
+  const unsigned int cut = sh.prefix, k_eq = sh.k_eq;
+  for (long base = 0; base < n; base += kSelThreads) {
+    const long e = base + tid;
+    bool gt = false, eq = false, causal = false;
+    if (e < n) {
+      const int i = (int)(e / nb), j = (int)(e % nb);
+      causal = j <= i;
+      if (causal) {
+        const unsigned int bits = __float_as_uint(sc[e]);
+        gt = bits > cut;
+        eq = bits == cut;
+      }
+    }
+    const unsigned int bal = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) sh.warp_cnt[warp] = __popc(bal);
+    __syncthreads();
+    unsigned int before = sh.running;
+    for (int w = 0; w < warp; ++w) before += sh.warp_cnt[w];
+    const unsigned int rank = before + __popc(bal & ((1u << lane) - 1u));
+    if (e < n) mk[e] = (uint8_t)(causal && (all || gt || (eq && rank < k_eq)) ? 1 : 0);
+    __syncthreads();
+    if (tid == 0) {
+      unsigned int t = 0;
+      for (int w = 0; w < kSelThreads / 32; ++w) t += sh.warp_cnt[w];
+      sh.running += t;
+    }
+    __syncthreads();
+  }
+}
+
+// ---- per row: force the diagonal into an empty row, compact the ascending list; one warp per row
+__global__ void compact_rows_kernel(uint8_t* __restrict__ mask, int n_maps, int nb, int32_t* __restrict__ counts,
+                                    int32_t* __restrict__ indices) {
+  const int lane = threadIdx.x & 31;
+  const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (w >= (long)n_maps * nb) return;
+  const int mp = (int)(w / nb), i = (int)(w % nb);
+  uint8_t* row = mask + ((size_t)mp * nb + i) * nb;
+  int32_t* irow = indices + ((size_t)mp * nb + i) * nb;
+  int cnt = 0;
+  for (int j0 = 0; j0 < nb; j0 += 32) {
+    const int j = j0 + lane;
+    const bool on = j <= i && row[j] != 0;
+    const unsigned int bal = __ballot_sync(0xffffffffu, on);
+    if (on) irow[cnt + __popc(bal & ((1u << lane) - 1u))] = j;
+    cnt += __popc(bal);
+  }
+  if (cnt == 0) {                          // a row-block must keep at least one key-block: its diagonal
+    if (lane == 0) { row[i] = 1; irow[0] = i; }
+    cnt = 1;
+  }
+  __syncwarp();
+  for (int j = cnt + lane; j < nb; j += 32) irow[j] = -1;
+  if (lane == 0) counts[(size_t)mp * nb + i] = cnt;
+}
+
+// ---- "Determine Sparse Pattern" ---------------------------------------------------------------
+// pooled last row: grid (Nb, n_heads), d threads.  Block j: mean of the last query block against the mean
+// of key block j; the last block uses the visible half.
+__global__ void last_row_pooled_kernel(const PooledArgs a) {
+  __shared__ float red[4];
+  const int j = blockIdx.x, slot = blockIdx.y, col = threadIdx.x;
+  const int h = a.heads.v[slot], g = h / a.group;
+  const int last = a.Nb - 1;
+  const __nv_bfloat16* q = a.q + (size_t)h * a.q_sh + (size_t)last * a.B * a.q_sn + col;
+  const __nv_bfloat16* k = a.k + (size_t)g * a.k_sh + (size_t)j * a.B * a.k_sn + col;
+  float acc = 0.f, denom;
+  if (j < last) {
+    float qsum = 0.f, ksum = 0.f;
+    for (int r = 0; r < a.B; ++r) {
+      qsum += __bfloat162float(q[(size_t)r * a.q_sn]);
+      ksum += __bfloat162float(k[(size_t)r * a.k_sn]);
+    }
+    acc = qsum * ksum;
+    denom = (float)a.B * (float)a.B;
+  } else {
+    float kcum = 0.f;
+    for (int r = 0; r < a.B; ++r) {
+      kcum += __bfloat162float(k[(size_t)r * a.k_sn]);
+      acc = fmaf(__bfloat162float(q[(size_t)r * a.q_sn]), kcum, acc);
+    }
+    denom = 0.5f * (float)a.B * (float)(a.B + 1);
+  }
+  acc = warp_sum(acc);
+  if ((col & 31) == 0) red[col >> 5] = acc;
+  __syncthreads();
+  if (col == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    a.pooled[(size_t)slot * a.Nb + j] = t * a.scale / denom;
+  }
+}
+
+// one CTA of 256 threads per head: softmax of the pooled last row, the two Jensen-Shannon distances, the decision
+__global__ void decide_pattern_kernel(const float* __restrict__ pooled_last, int nb, const float* __restrict__ pivot_rows,
+                                      HeadTable row_of_head, float delta, float tau, int32_t* __restrict__ pattern,
+                                      float* __restrict__ dist) {
+  __shared__ float red[8];
+  __shared__ float bc[2];
+  const int slot = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* z = pooled_last + (size_t)slot * nb;
+  const int prow = row_of_head.v[slot];
+  const float* at = prow >= 0 ? pivot_rows + (size_t)prow * nb : nullptr;
+  auto block_reduce = [&](float v, bool is_max) {
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    if (tid == 0) {
+      float t = red[0];
+      for (int w = 1; w < (int)(blockDim.x >> 5); ++w) t = is_max ? fmaxf(t, red[w]) : t + red[w];
+      bc[0] = t;
+    }
+    __syncthreads();
+    return bc[0];
+  };
+  float m = -CUDART_INF_F;
+  for (int j = tid; j < nb; j += blockDim.x) m = fmaxf(m, z[j]);
+  m = block_reduce(m, true);
+  float s = 0.f;
+  for (int j = tid; j < nb; j += blockDim.x) s += expf(z[j] - m);
+  s = block_reduce(s, false);
+  const float inv = 1.f / s, u = 1.f / (float)nb;
+  // JSD(p || q) = 1/2 sum p ln(p/m) + 1/2 sum q ln(q/m), m = (p + q)/2, 0 ln 0 = 0
+  float js_u = 0.f, js_a = 0.f;
+  for (int j = tid; j < nb; j += blockDim.x) {
+    const float p = expf(z[j] - m) * inv;
+    {
+      const float mm = 0.5f * (p + u);
+      js_u += (p > 0.f ? p * logf(p / mm) : 0.f) + u * logf(u / mm);
+    }
+    if (at) {
+      const float q = at[j], mm = 0.5f * (p + q);
+      js_a += (p > 0.f ? p * logf(p / mm) : 0.f) + (q > 0.f ? q * logf(q / mm) : 0.f);
+    }
+  }
+  js_u = block_reduce(js_u, false);
+  js_a = block_reduce(js_a, false);
+  if (tid == 0) {
+    const float d_sparse = sqrtf(fmaxf(0.5f * js_u, 0.f));
+    const float d_sim = at ? sqrtf(fmaxf(0.5f * js_a, 0.f)) : CUDART_INF_F;
+    pattern[slot] = (d_sparse < delta && d_sim < tau) ? 0 : 1;
+    if (dist) { dist[2 * slot] = d_sparse; dist[2 * slot + 1] = d_sim; }
+  }
+}
+
+}  // namespace
+
+size_t pooled_scratch_floats(int n_heads, int Nb, int d) { return (size_t)n_heads * Nb * (2 * (size_t)d + 1); }
+
+cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s) {
+  if (a.n_heads == 0) return cudaSuccess;
+  block_means_kernel<<<dim3(a.Nb, a.n_heads), a.d, 0, s>>>(a);
+  pooled_logits_kernel<<<dim3(a.Nb, a.n_heads), 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
+                                       uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
+                                       cudaStream_t s) {
+  if (n_maps == 0) return cudaSuccess;
+  const long rows = (long)n_maps * nb;
+  pooled_softmax_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(pooled, n_maps, nb, scores, last_row);
+  cudaError_t e = cudaFuncSetAttribute(global_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)sizeof(SelShared));
+  if (e != cudaSuccess) return e;
+  global_select_kernel<<<n_maps, kSelThreads, sizeof(SelShared), s>>>(scores, nb, gamma, mask);
+  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,
+                                     float delta, float tau, int32_t* pattern, float* dist, cudaStream_t s) {
+  if (a.n_heads == 0) return cudaSuccess;
+  last_row_pooled_kernel<<<dim3(a.Nb, a.n_heads), a.d, 0, s>>>(a);     // a.pooled: [n_heads, Nb] here
+  decide_pattern_kernel<<<a.n_heads, 256, 0, s>>>(a.pooled, a.Nb, pivot_rows, row_of_head, delta, tau, pattern, dist);
+  return cudaGetLastError();
+}
+
+}  // namespace sp

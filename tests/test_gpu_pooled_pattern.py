@@ -1,0 +1,155 @@
+"""GPU parity of the paper-literal pattern construction and decision (block-averaged QK values,
+global cumulative cut, Jensen-Shannon decision) against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pooled_pattern_oracle as ppo
+from paper_2505_19578_b200 import synth
+from tests import _parity as par
+
+pytestmark = pytest.mark.gpu
+
+POOLED_ATOL = 2e-5     # fp32 block means and dot products of bf16 data, logits of order 1..30
+SCORE_BAND = 2e-5      # an entry may flip only if the oracle's cumulative score at it is this close to gamma
+DIV_ATOL = 2e-6        # Jensen-Shannon divergences (squared distances) from fp32 distributions;
+                       # the square root amplifies rounding near zero, so the squares are compared
+DIST_MARGIN = 2e-3     # a decision is checked when both distances are this far from their thresholds
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2505_19578_b200 import binding as b, build
+    build.build()
+    return b
+
+
+def _oracle_cut(At, g):
+    """Oracle result plus, per block, the cumulative normalised score at which it enters the order."""
+    res = ppo.construct_pivotal_pattern(At, g)
+    Nb = At.shape[0]
+    flat = (res["scores"] / res["scores"].sum()).reshape(-1)
+    idx = np.flatnonzero(np.tril(np.ones((Nb, Nb), bool)).reshape(-1))
+    order = idx[np.argsort(-flat[idx], kind="stable")]
+    cum_at = np.full(Nb * Nb, np.inf)
+    cum_at[order] = np.cumsum(flat[order])
+    return res, cum_at.reshape(Nb, Nb), flat.reshape(Nb, Nb)
+
+
+@pytest.mark.parametrize("name,seq,gamma", [("llama8b_32k", 4096, 0.9), ("tiny", 2048, 0.8), ("qwen7b_64k", 4096, 0.95)])
+def test_pooled_logits_and_pattern_match_oracle(binding, name, seq, gamma):
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=3)
+    cfg = L["cfg"]
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    heads = list(L["pivot_heads"]) + [h for h in range(cfg.n_q_heads) if h not in L["pivot_heads"]][:1]
+    ctx = binding.Context()
+    q, k = L["q"].cuda(), L["k"].cuda()
+    pooled = torch.full((len(heads), Nb, Nb), float("nan"), device="cuda")
+    ctx.sp_pooled_logits(q, k, heads, B, pooled)
+    mask = torch.full((len(heads), Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+    counts = torch.full((len(heads), Nb), -5, dtype=torch.int32, device="cuda")
+    idx = torch.full((len(heads), Nb, Nb), -5, dtype=torch.int32, device="cuda")
+    last = torch.full((len(heads), Nb), float("nan"), device="cuda")
+    ctx.sp_pattern_from_pooled(pooled, gamma, mask, counts, idx, last_row_out=last)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    Q, K = par.f64(L["q"]), par.f64(L["k"])
+    g = par.gamma32(gamma)
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    for t, h in enumerate(heads):
+        At = ppo.pooled_logits(Q[h], K[h // G], B)
+        got = pooled[t].cpu().numpy().astype(np.float64)
+        tri = np.tril(np.ones((Nb, Nb), bool))
+        assert np.all(got[~tri] == -np.inf)
+        np.testing.assert_allclose(got[tri], At[tri], rtol=0, atol=POOLED_ATOL)
+        res, cum_at, flat = _oracle_cut(At, g)
+        np.testing.assert_allclose(last[t].cpu().numpy(), res["a_last"], rtol=0, atol=1e-6)
+        m = mask[t].cpu().numpy()
+        assert np.all(m[~tri] == 0) and np.all(m.sum(axis=1) >= 1)
+        # entries may differ from the oracle only next to the cut (or as a forced diagonal that follows from it)
+        diff = np.argwhere(m != res["mask"])
+        for i, j in diff:
+            near = abs(cum_at[i, j] - g) <= SCORE_BAND or abs(cum_at[i, j] - flat[i, j] - g) <= SCORE_BAND
+            forced = i == j and (m[i].sum() == 1 or res["mask"][i].sum() == 1)
+            assert near or forced, (h, i, j, cum_at[i, j], g)
+        assert len(diff) <= 4
+        # lists and counts describe the mask
+        c, ix = counts[t].cpu().numpy(), idx[t].cpu().numpy()
+        for i in range(Nb):
+            sel = np.flatnonzero(m[i])
+            assert c[i] == len(sel) and np.array_equal(ix[i, :c[i]], sel) and np.all(ix[i, c[i]:] == -1)
+
+
+def test_pattern_from_pooled_exact_cases(binding):
+    # equal scores inside a row (ties go to the smaller index), forced diagonals, unreachable gamma; the
+    # gammas stay clear of the cumulative sums 1/8, 3/16, 1/4, ... where fp32 scores could fall either way
+    Nb = 8
+    At = np.where(np.tril(np.ones((Nb, Nb), bool)), 0.0, -np.inf).astype(np.float32)     # uniform rows: scores 1/(i+1)
+    ctx = binding.Context()
+    pooled = torch.from_numpy(np.stack([At, At])).cuda()
+    for gamma in (0.15, 0.2, 0.26, 0.6, 0.9, 1e-6, 1.5):
+        mask = torch.zeros(2, Nb, Nb, dtype=torch.uint8, device="cuda")
+        counts = torch.zeros(2, Nb, dtype=torch.int32, device="cuda")
+        idx = torch.zeros(2, Nb, Nb, dtype=torch.int32, device="cuda")
+        ctx.sp_pattern_from_pooled(pooled, gamma, mask, counts, idx)
+        torch.cuda.synchronize()
+        res = ppo.construct_pivotal_pattern(At.astype(np.float64), par.gamma32(gamma))
+        for t in range(2):
+            assert np.array_equal(mask[t].cpu().numpy(), res["mask"]), gamma
+            assert np.array_equal(counts[t].cpu().numpy(), res["mask"].sum(axis=1))
+
+
+@pytest.mark.parametrize("name,seq", [("llama8b_32k", 4096), ("qwen7b_64k", 2048)])
+def test_determine_pattern_matches_oracle(binding, name, seq):
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=5)
+    cfg = L["cfg"]
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    piv = list(L["pivot_heads"])
+    ctx = binding.Context()
+    q, k = L["q"].cuda(), L["k"].cuda()
+    pooled = torch.empty(len(piv), Nb, Nb, device="cuda")
+    ctx.sp_pooled_logits(q, k, piv, B, pooled)
+    mask = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device="cuda")
+    counts = torch.empty(len(piv), Nb, dtype=torch.int32, device="cuda")
+    idx = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device="cuda")
+    last = torch.empty(len(piv), Nb, device="cuda")
+    ctx.sp_pattern_from_pooled(pooled, 0.9, mask, counts, idx, last_row_out=last)
+    first = {}
+    for t, p in enumerate(piv):
+        first.setdefault(L["cluster_map"][p], t)
+    heads = list(range(cfg.n_q_heads))
+    rows = [first.get(L["cluster_map"][h], -1) for h in heads]
+    rows[-1] = -1                                             # one head without a pivotal representative
+    pat = torch.full((len(heads),), -1, dtype=torch.int32, device="cuda")
+    dist = torch.full((len(heads), 2), float("nan"), device="cuda")
+    Q, K = par.f64(L["q"]), par.f64(L["k"])
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    a_tilde = [ppo.construct_pivotal_pattern(ppo.pooled_logits(Q[p], K[p // G], B), 0.9)["a_last"] for p in piv]
+    ref = []
+    for h, r in zip(heads, rows):
+        a_hat = ppo.last_block_distribution(Q[h], K[h // G], B)
+        ref.append(ppo.determine_pattern(a_hat, a_tilde[r] if r >= 0 else None, 0.3, 0.2))
+    # thresholds that split the heads: medians of the oracle's distances
+    delta = float(np.median([r[1] for r in ref])) + 1e-3
+    tau = float(np.median([r[2] for r in ref if np.isfinite(r[2])])) + 1e-3
+    ctx.sp_determine_pattern(q, k, heads, B, last, rows, delta, tau, pat, dist_out=dist)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    got_p, got_d = pat.cpu().numpy(), dist.cpu().numpy()
+    n_shared = 0
+    for x, (h, r) in enumerate(zip(heads, rows)):
+        _, ds, dm = ref[x]
+        assert float(got_d[x, 0]) ** 2 == pytest.approx(ds * ds, abs=DIV_ATOL)
+        if np.isfinite(dm):
+            assert float(got_d[x, 1]) ** 2 == pytest.approx(dm * dm, abs=DIV_ATOL)
+        else:
+            assert np.isinf(got_d[x, 1])
+        want = 0 if (ds < delta and dm < tau) else 1
+        if min(abs(ds - delta), abs(dm - tau)) > DIST_MARGIN:     # away from the thresholds the decision is fixed
+            assert got_p[x] == want
+        n_shared += int(got_p[x] == 0)
+    assert 0 < n_shared < len(heads)                                # the thresholds really split the heads
+    # a pivot compared with its own representative: distance 0
+    for t, p in enumerate(piv):
+        if rows[p] == t:
+            assert got_d[p, 1] <= 2e-3
