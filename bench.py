@@ -294,6 +294,41 @@ def run_ours(args):
         dense_ms = d0.elapsed_time(d1) / 2
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
+    literal = None
+    if rank == 0 and not args.no_literal:
+        pooled = torch.empty(len(piv), Nb, Nb, device=dev)
+        lm = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device=dev)
+        lc = torch.empty(len(piv), Nb, dtype=torch.int32, device=dev)
+        li = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device=dev)
+        last = torch.empty(len(piv), Nb, device=dev)
+        pat = torch.empty(cfg.n_q_heads, dtype=torch.int32, device=dev)
+        rows = [first_pivot_of.get(cm[h], -1) if cm[h] >= 0 else -1 for h in range(cfg.n_q_heads)]
+
+        def literal_step(e):
+            e[0].record(stream)
+            ctx.sp_pooled_logits(q, k, piv, B, pooled, stream=stream)
+            e[1].record(stream)
+            ctx.sp_pattern_from_pooled(pooled, gamma, lm, lc, li, last_row_out=last, stream=stream)
+            e[2].record(stream)
+            ctx.sp_determine_pattern(q, k, list(range(cfg.n_q_heads)), B, last, rows, 0.3, 0.2, pat, stream=stream)
+            e[3].record(stream)
+
+        le = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        literal_step(le)
+        torch.cuda.synchronize()
+        literal_step(le)
+        torch.cuda.synchronize()
+        inter = (lm & pm).sum(dim=(1, 2)).float()
+        union = (lm | pm).sum(dim=(1, 2)).float()
+        literal = {
+            "pooled_logits_ms": le[0].elapsed_time(le[1]), "pattern_from_pooled_ms": le[1].elapsed_time(le[2]),
+            "determine_pattern_ms": le[2].elapsed_time(le[3]),
+            "mask_density_per_pivot": {int(p): float(lc[t].sum().item()) / tiles_causal for t, p in enumerate(piv)},
+            "jaccard_with_mass_mask_per_pivot": {int(p): float(inter[t] / union[t]) for t, p in enumerate(piv)},
+            "heads_shared_pivot_at_delta0.3_tau0.2": int((pat == 0).sum().item()),
+        }
+
     # ---- end to end through the C ABI with host buffers: H2D of q,k,v, the layer, D2H of the output
     hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
@@ -368,6 +403,7 @@ def run_ours(args):
         "roofline": roofline,
         "e2e": {"value": layers * F / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "paper_literal_pattern": literal,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -397,6 +433,7 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-literal", action="store_true", help="skip the paper-literal pattern construction leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:

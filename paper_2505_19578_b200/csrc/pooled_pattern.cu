@@ -13,7 +13,7 @@
 // of Q and of K, so the map needs no pass over the tiles: block means of Q and K
 // (one read of the two tensors), one small product per block, and the diagonal
 // block (only its visible half is averaged) through a running key prefix sum.
-// The global cut is a radix select on the score bits with float64 bin sums
+// The global cut is a radix select on the score bits with exact fixed-point bin sums
 // (three passes of 11 + 11 + 10 bits), followed by an ordered pass that breaks
 // ties towards the smaller flattened index.  All of it is HBM- and latency-sized
 // work (a few MB per head).
@@ -111,10 +111,15 @@ __global__ void pooled_softmax_kernel(const float* __restrict__ pooled, int n_ma
 constexpr int kSelThreads = 1024;
 constexpr int kBins = 2048;
 
+// Bin sums are kept in 2^-60 fixed point: integer additions commute, so the cut does not depend on
+// the order in which the threads arrive (normalised scores sum to 1: no overflow in 64 bits).
+constexpr double kFix = 1152921504606846976.0;   // 2^60
+
 struct SelShared {
   unsigned int count[kBins];
-  double sum[kBins];
-  double total, cum_above;
+  unsigned long long sum[kBins];
+  double total;
+  unsigned long long cum_above;
   unsigned int prefix, k_eq, running, select_all;
   unsigned int warp_cnt[kSelThreads / 32];
 };
@@ -124,59 +129,62 @@ __global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float*
   extern __shared__ unsigned char sel_raw[];
   SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
   const int mp = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kWarps = kSelThreads / 32;
   const float* sc = scores + (size_t)mp * nb * nb;
   uint8_t* mk = mask + (size_t)mp * nb * nb;
-  const long n = (long)nb * nb;
+
+  // Rows are dealt to the warps round-robin (balanced: long and short rows alternate), lanes run
+  // along a row's existing blocks j <= i.
 
   // total of the map (each row sums to 1 up to rounding), float64
-  if (tid == 0) { sh.total = 0.0; sh.cum_above = 0.0; sh.prefix = 0u; sh.select_all = 0u; sh.running = 0u; }
+  if (tid == 0) { sh.total = 0.0; sh.cum_above = 0ull; sh.prefix = 0u; sh.select_all = 0u; sh.running = 0u; sh.k_eq = 0u; }
   __syncthreads();
   {
     double t = 0.0;
-    for (long e = tid; e < n; e += kSelThreads) {
-      const int i = (int)(e / nb), j = (int)(e % nb);
-      if (j <= i) t += (double)sc[e];
-    }
+    for (int i = warp; i < nb; i += kWarps)
+      for (int j = lane; j <= i; j += 32) t += (double)sc[(size_t)i * nb + j];
     for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
     if (lane == 0) atomicAdd(&sh.total, t);
   }
   __syncthreads();
-  const double inv_total = 1.0 / sh.total;
+  const double inv_total = kFix / sh.total;
+  const unsigned long long gamma_fx = gamma >= 4.0 ? ~0ull : __double2ull_rn(gamma * kFix);
 
   // radix select, most significant digit first: digits of 11, 11, 10 bits
   const int shift[3] = {21, 10, 0};
-  const unsigned int dmask[3] = {0x7FFu, 0x7FFu, 0x3FFu};
+  const int width[3] = {11, 11, 10};
   for (int pass = 0; pass < 3 && !sh.select_all; ++pass) {
-    for (int b = tid; b < kBins; b += kSelThreads) { sh.count[b] = 0u; sh.sum[b] = 0.0; }
+    for (int b = tid; b < kBins; b += kSelThreads) { sh.count[b] = 0u; sh.sum[b] = 0ull; }
     __syncthreads();
     const unsigned int prefix = sh.prefix;
-    const int above = shift[pass] + (pass == 0 ? 11 : (pass == 1 ? 11 : 10));   // bits above this digit
-    for (long e = tid; e < n; e += kSelThreads) {
-      const int i = (int)(e / nb), j = (int)(e % nb);
-      if (j > i) continue;
-      const unsigned int bits = __float_as_uint(sc[e]);
-      if (pass > 0 && (bits >> above) != prefix) continue;
-      const unsigned int dgt = (bits >> shift[pass]) & dmask[pass];
-      atomicAdd(&sh.count[dgt], 1u);
-      atomicAdd(&sh.sum[dgt], (double)sc[e] * inv_total);
+    const int above = shift[pass] + width[pass];          // bits above this digit
+    const unsigned int dmask = (1u << width[pass]) - 1u;
+    for (int i = warp; i < nb; i += kWarps) {
+      for (int j = lane; j <= i; j += 32) {
+        const float v = sc[(size_t)i * nb + j];
+        const unsigned int bits = __float_as_uint(v);
+        if (pass > 0 && (bits >> above) != prefix) continue;
+        const unsigned int dgt = (bits >> shift[pass]) & dmask;
+        atomicAdd(&sh.count[dgt], 1u);
+        atomicAdd(&sh.sum[dgt], __double2ull_rn((double)v * inv_total));
+      }
     }
     __syncthreads();
     if (tid == 0) {
-      double cum = sh.cum_above;
-      int b = (int)dmask[pass];
+      unsigned long long cum = sh.cum_above;
+      int b = (int)dmask;
       bool found = false;
       int lowest = -1;                    // lowest non-empty digit seen
-      double cum_before_lowest = cum;
+      unsigned long long cum_before_lowest = cum;
       for (; b >= 0; --b) {
         if (sh.count[b] == 0u) continue;
         lowest = b;
         cum_before_lowest = cum;
-        if (cum + sh.sum[b] >= gamma) { found = true; break; }
+        if (cum + sh.sum[b] >= gamma_fx) { found = true; break; }
         cum += sh.sum[b];
       }
       if (!found && pass > 0 && lowest >= 0) {
-        // the digit above said the cut lies in this group; its members were summed in another order
-        // and fall short by rounding: the cut is the group's smallest value
+        // cannot happen with exact integer sums; kept as a guard: the cut is the group's smallest value
         found = true;
         b = lowest;
         cum = cum_before_lowest;
@@ -185,14 +193,14 @@ __global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float*
         sh.select_all = 1u;                       // the scores never reach gamma: every block that exists
       } else {
         sh.cum_above = cum;
-        sh.prefix = (prefix << (pass == 2 ? 10 : 11)) | (unsigned int)b;
+        sh.prefix = (prefix << width[pass]) | (unsigned int)b;
         if (pass == 2) {
           // prefix is now the bit pattern of the cut value; how many of its copies are needed
-          const double v = (double)__uint_as_float(sh.prefix) * inv_total;
+          const unsigned long long v = __double2ull_rn((double)__uint_as_float(sh.prefix) * inv_total);
           unsigned int k = 0;
-          double c = cum;
+          unsigned long long c = cum;
           const unsigned int n_eq = sh.count[b];
-          do { c += v; ++k; } while (c < gamma && k < n_eq);
+          do { c += v; ++k; } while (c < gamma_fx && k < n_eq);
           sh.k_eq = k;
         }
       }
@@ -200,32 +208,43 @@ __global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float*
     __syncthreads();
   }
 
-  // ordered marking: everything above the cut value, and the first k_eq copies of it in row-major order
+  // marking: everything above the cut value, and the first k_eq copies of it in row-major order.
+  // Groups of kWarps consecutive rows, one row per warp: count the copies per row, prefix over the
+  // group's rows, then mark.
   const bool all = sh.select_all != 0u;
   const unsigned int cut = sh.prefix, k_eq = sh.k_eq;
-  for (long base = 0; base < n; base += kSelThreads) {
-    const long e = base + tid;
-    bool gt = false, eq = false, causal = false;
-    if (e < n) {
-      const int i = (int)(e / nb), j = (int)(e % nb);
-      causal = j <= i;
-      if (causal) {
-        const unsigned int bits = __float_as_uint(sc[e]);
-        gt = bits > cut;
-        eq = bits == cut;
+  for (int i0 = 0; i0 < nb; i0 += kWarps) {
+    const int i = i0 + warp;
+    unsigned int n_eq_row = 0;
+    if (i < nb && !all)
+      for (int j0 = 0; j0 <= i; j0 += 32) {
+        const int j = j0 + lane;
+        const bool eq = j <= i && __float_as_uint(sc[(size_t)i * nb + j]) == cut;
+        n_eq_row += __popc(__ballot_sync(0xffffffffu, eq));
+      }
+    if (lane == 0) sh.warp_cnt[warp] = n_eq_row;
+    __syncthreads();
+    unsigned int rank0 = sh.running;
+    for (int w = 0; w < warp; ++w) rank0 += sh.warp_cnt[w];
+    if (i < nb) {
+      for (int j0 = 0; j0 < nb; j0 += 32) {
+        const int j = j0 + lane;
+        bool on = false;
+        unsigned int bal = 0u;
+        const bool causal = j <= i;
+        unsigned int bits = 0u;
+        if (causal) bits = __float_as_uint(sc[(size_t)i * nb + j]);
+        const bool eq = causal && !all && bits == cut;
+        bal = __ballot_sync(0xffffffffu, eq);
+        if (causal) on = all || bits > cut || (eq && rank0 + __popc(bal & ((1u << lane) - 1u)) < k_eq);
+        if (j < nb) mk[(size_t)i * nb + j] = (uint8_t)(on ? 1 : 0);
+        rank0 += __popc(bal);
       }
     }
-    const unsigned int bal = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) sh.warp_cnt[warp] = __popc(bal);
-    __syncthreads();
-    unsigned int before = sh.running;
-    for (int w = 0; w < warp; ++w) before += sh.warp_cnt[w];
-    const unsigned int rank = before + __popc(bal & ((1u << lane) - 1u));
-    if (e < n) mk[e] = (uint8_t)(causal && (all || gt || (eq && rank < k_eq)) ? 1 : 0);
     __syncthreads();
     if (tid == 0) {
       unsigned int t = 0;
-      for (int w = 0; w < kSelThreads / 32; ++w) t += sh.warp_cnt[w];
+      for (int w = 0; w < kWarps; ++w) t += sh.warp_cnt[w];
       sh.running += t;
     }
     __syncthreads();
