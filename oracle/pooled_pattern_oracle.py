@@ -22,6 +22,13 @@ What is defined here, step by step as the paper states it:
                              d_sim = sqrt(JSD(a^ || a~)); shared pivot iff
                              d_sparse < delta and d_sim < tau, else vertical-slash.
 
+  * vertical_slash_scores, search_vertical_slash_pattern  Algorithm "Search Vertical Slash
+                             Pattern": A^ = softmax(Q^ K^T / sqrt(d)) for the last block
+                             of queries, sums along the vertical (per key) and slash (per
+                             query-minus-key offset) directions, each normalised, sorted and
+                             cut at gamma, union of the selected lines turned into a block
+                             mask.
+
 Readings taken where the paper is silent (also listed in the design notes):
   * causal: a block above the diagonal is never computed (average −inf); the
     average of the diagonal block runs over its visible entries (key <= query);
@@ -33,7 +40,11 @@ Readings taken where the paper is silent (also listed in the design notes):
   * sort descending, ties to the smaller flattened (row-major) index, ">= gamma";
   * a row-block left without any selected block would make the masked softmax
     of its rows undefined: it receives its diagonal block (forced, counted);
-  * Jensen-Shannon divergence with natural logarithms, 0 log 0 = 0.
+  * Jensen-Shannon divergence with natural logarithms, 0 log 0 = 0;
+  * vertical-slash: Q^ is the last block of queries; a slash line is the set of (query r, key c)
+    with r - c = o for an offset o >= 0; index_to_mask computes a block if it contains a selected
+    key column or is crossed by a selected slash line (and lies on or below the diagonal); an empty
+    row-block receives its diagonal block as above.
 
 Everything is numpy float64 on the bf16-rounded inputs.  Pins:
 tests/test_pooled_oracle_pins.py.  Parity with the authors' implementation is
@@ -52,6 +63,9 @@ __all__ = [
     "last_block_distribution",
     "js_distance",
     "determine_pattern",
+    "cumulative_select",
+    "vertical_slash_scores",
+    "search_vertical_slash_pattern",
 ]
 
 
@@ -162,3 +176,63 @@ def determine_pattern(a_hat, a_tilde, delta: float, tau: float):
     d_sim = js_distance(a_hat, a_tilde) if a_tilde is not None else math.inf
     pattern = "shared_pivot" if (d_sparse < delta and d_sim < tau) else "vertical_slash"
     return pattern, d_sparse, d_sim
+
+
+def cumulative_select(a, gamma: float):
+    """Minimum prefix of the descending order of the non-negative vector a (normalised by its sum)
+    whose scores sum to >= gamma; equal scores go to the smaller index; everything if never reached.
+    Returns (selected bool [len(a)], K)."""
+    a = np.asarray(a, dtype=np.float64)
+    flat = a / a.sum()
+    order = np.argsort(-flat, kind="stable")
+    cum = np.cumsum(flat[order])
+    hit = np.flatnonzero(cum >= gamma)
+    K = int(hit[0]) + 1 if hit.size else len(order)
+    sel = np.zeros(len(a), dtype=bool)
+    sel[order[:K]] = True
+    return sel, K
+
+
+def vertical_slash_scores(Qh, Kg, B: int):
+    """A^ = softmax(Q^ K^T / sqrt(d)), causal, for the last block of queries; returns
+    (a_v [N], a_s [N]): its sums per key column and per offset o = query - key (o >= 0), unnormalised
+    (both sum to the number of rows of Q^)."""
+    Qh = np.asarray(Qh, dtype=np.float64)
+    Kg = np.asarray(Kg, dtype=np.float64)
+    N, d = Qh.shape
+    Nb = (N + B - 1) // B
+    r0 = (Nb - 1) * B
+    S = (Qh[r0:N] @ Kg.T) / math.sqrt(d)
+    rows = np.arange(r0, N)[:, None]
+    cols = np.arange(N)[None, :]
+    S = np.where(cols <= rows, S, -np.inf)
+    P = np.exp(S - S.max(axis=1, keepdims=True))
+    P /= P.sum(axis=1, keepdims=True)
+    a_v = P.sum(axis=0)
+    a_s = np.zeros(N)
+    for x in range(P.shape[0]):                      # row r0 + x: offset o = r - c
+        r = r0 + x
+        a_s[:r + 1] += P[x, r::-1]                   # c = r - o for o = 0..r
+    return a_v, a_s
+
+
+def search_vertical_slash_pattern(Qh, Kg, gamma: float, B: int):
+    """Algorithm "Search Vertical Slash Pattern" -> dict(mask u8 [Nb, Nb], sel_v, sel_s, K_v, K_s, forced)."""
+    N = np.asarray(Qh).shape[0]
+    Nb = (N + B - 1) // B
+    a_v, a_s = vertical_slash_scores(Qh, Kg, B)
+    sel_v, K_v = cumulative_select(a_v, gamma)
+    sel_s, K_s = cumulative_select(a_s, gamma)
+    mask = np.zeros((Nb, Nb), dtype=np.uint8)
+    col_block = np.array([sel_v[j * B:(j + 1) * B].any() for j in range(Nb)])
+    for i in range(Nb):
+        for j in range(i + 1):
+            lo = max((i - j) * B - (B - 1), 0)       # offsets r - c reachable inside block (i, j)
+            hi = min((i - j) * B + (B - 1), N - 1)
+            if col_block[j] or sel_s[lo:hi + 1].any():
+                mask[i, j] = 1
+    forced = [i for i in range(Nb) if mask[i].sum() == 0]
+    for i in forced:
+        mask[i, i] = 1
+    return {"mask": mask, "sel_v": sel_v, "sel_s": sel_s, "K_v": K_v, "K_s": K_s, "forced": forced,
+            "a_v": a_v, "a_s": a_s}

@@ -171,3 +171,96 @@ def test_determine_pattern_thresholds_are_strict():
     assert ppo.determine_pattern(a, None, 1.0, 1.0)[0] == "vertical_slash"        # no pivotal representative yet
     pat, d1, d2 = ppo.determine_pattern(a, b, 0.3, 0.2)
     assert (d1, d2) == (pytest.approx(ds), pytest.approx(dsim))
+
+
+# ------------------------------------------------------------------ vertical-slash search
+
+def test_vertical_slash_scores_equal_scalar_brute_force():
+    N, d, B = 40, 4, 16
+    Q, K = _rand(N, d, 11)
+    a_v, a_s = ppo.vertical_slash_scores(Q, K, B)
+    r0 = 32
+    ev, es = [0.0] * N, [0.0] * N
+    for r in range(r0, N):
+        logits = [sum(Q[r, t] * K[c, t] for t in range(d)) / math.sqrt(d) for c in range(r + 1)]
+        mx = max(logits)
+        den = sum(math.exp(x - mx) for x in logits)
+        for c in range(r + 1):
+            p = math.exp(logits[c] - mx) / den
+            ev[c] += p
+            es[r - c] += p
+    np.testing.assert_allclose(a_v, ev, atol=1e-13)
+    np.testing.assert_allclose(a_s, es, atol=1e-13)
+    assert a_v.sum() == pytest.approx(N - r0) and a_s.sum() == pytest.approx(N - r0)
+
+
+def test_vertical_slash_closed_forms():
+    # Q = 0: every visible key of row r has probability 1/(r+1); vertical and slash sums coincide by symmetry
+    N, d, B = 64, 4, 16
+    Q = np.zeros((N, d)); K = np.random.default_rng(1).standard_normal((N, d))
+    a_v, a_s = ppo.vertical_slash_scores(Q, K, B)
+    rows = range(N - B, N)
+    for c in (0, 10, 47, 50, 63):
+        assert a_v[c] == pytest.approx(sum(1.0 / (r + 1) for r in rows if r >= c))
+    for o in (0, 5, 48, 60, 63):
+        assert a_s[o] == pytest.approx(sum(1.0 / (r + 1) for r in rows if r >= o))
+    # one key dominates every row -> that column carries all the vertical mass; the slash mass of row r sits at r - c0
+    c0 = 7
+    Q = np.ones((N, d)); K = np.zeros((N, d)); K[c0] = 30.0
+    a_v, a_s = ppo.vertical_slash_scores(Q, K, B)
+    assert a_v[c0] == pytest.approx(B, rel=1e-9)
+    for r in rows:
+        assert a_s[r - c0] == pytest.approx(1.0, rel=1e-9)
+
+
+def test_cumulative_select_minimal_ties_and_extremes():
+    a = np.array([0.1, 0.4, 0.1, 0.2, 0.2])
+    sel, K = ppo.cumulative_select(a, 0.6)
+    assert K == 2 and sel.tolist() == [False, True, False, True, False]      # 0.4 + first of the two 0.2
+    sel, K = ppo.cumulative_select(a, 0.6 + 1e-12)
+    assert K == 3 and sel.tolist() == [False, True, False, True, True]
+    sel, K = ppo.cumulative_select(a, 1e-9)
+    assert K == 1 and sel[1]
+    sel, K = ppo.cumulative_select(a, 2.0)
+    assert K == 5 and sel.all()
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        a = rng.random(7) ** 3
+        g = float(rng.uniform(0.1, 0.95))
+        sel, K = ppo.cumulative_select(a, g)
+        f = a / a.sum()
+        assert f[sel].sum() >= g - 1e-15
+        for k in range(K):
+            for sub in itertools.combinations(range(7), k):
+                assert f[list(sub)].sum() < g
+
+
+def test_vertical_slash_mask_geometry():
+    # planted lines: a heavy key column c0 and the slash at offset o0 must light exactly the blocks they cross
+    N, d, B = 128, 8, 16
+    Nb = N // B
+    rng = np.random.default_rng(4)
+    Q, K = rng.standard_normal((N, d)) * 0.01, rng.standard_normal((N, d)) * 0.01
+    res = ppo.search_vertical_slash_pattern(Q, K, 0.5, B)
+    m = res["mask"]
+    assert np.all(np.triu(m, 1) == 0) and np.all(m.sum(axis=1) >= 1)
+    for i in range(Nb):
+        for j in range(i + 1):
+            want = res["sel_v"][j * B:(j + 1) * B].any()
+            for r in range(i * B, (i + 1) * B):
+                for c in range(j * B, (j + 1) * B):
+                    if r - c >= 0 and res["sel_s"][r - c]:
+                        want = True
+            if i in res["forced"] and i == j:
+                want = True
+            assert m[i, j] == int(want)
+    # masks grow with gamma
+    prev = None
+    for g in (0.2, 0.5, 0.8, 0.95):
+        r = ppo.search_vertical_slash_pattern(Q, K, g, B)
+        mm = r["mask"].copy()
+        for i in r["forced"]:
+            mm[i, i] = 0
+        if prev is not None:
+            assert np.all(prev <= mm)
+        prev = mm
