@@ -282,6 +282,26 @@ int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
                          const int32_t* row_of_head, float delta, float tau, int32_t* pattern_out,
                          float* dist_out, void* stream);
 
+/*
+ * sp_vertical_slash_pattern - Algorithm "Search Vertical Slash Pattern" (the
+ *   fallback pattern of heads that do not share a pivotal pattern): A^ =
+ *   softmax(Q^ K^T / sqrt(head_dim)), causal, for Q^ = the last block of queries;
+ *   its sums per key column (vertical) and per offset o = query - key >= 0 (slash),
+ *   each normalised, ordered descending (equal scores: smaller index first) and cut
+ *   at the minimum budget whose scores sum to >= gamma; the union of the selected
+ *   lines is turned into a block mask: block (i, j), j <= i, is computed if
+ *   key-block j contains a selected column or a selected offset lies in
+ *   [(i-j) block - (block-1), (i-j) block + (block-1)].  A row-block left empty
+ *   receives its diagonal block.  head_dim 128 and block 128 only.
+ *     heads host [n_heads]; mask_out / counts_out / indices_out as for
+ *     sp_block_mask_from_importance (all required), directly usable by
+ *     sp_block_sparse_attn; sel_v_out, sel_s_out device u8 [n_heads, seq] or NULL:
+ *     the selected columns and offsets.
+ */
+int sp_vertical_slash_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads,
+                              int n_heads, float gamma, int block, uint8_t* mask_out, int32_t* counts_out,
+                              int32_t* indices_out, uint8_t* sel_v_out, uint8_t* sel_s_out, void* stream);
+
 /* Which attention kernel the context launches: 0 = tensor-core kernels
  * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V

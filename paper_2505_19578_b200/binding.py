@@ -30,7 +30,7 @@ EXPORTS = (
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
-    "sp_determine_pattern",
+    "sp_determine_pattern", "sp_vertical_slash_pattern",
 )
 
 
@@ -76,6 +76,7 @@ def load() -> ctypes.CDLL:
     lib.sp_pooled_logits.argtypes = [P, T, T, IP, I, I, P, P]
     lib.sp_pattern_from_pooled.argtypes = [P, P, I, I, F, P, P, P, P, P]
     lib.sp_determine_pattern.argtypes = [P, T, T, IP, I, I, P, IP, F, F, P, P, P]
+    lib.sp_vertical_slash_pattern.argtypes = [P, T, T, IP, I, F, I, P, P, P, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
@@ -208,6 +209,13 @@ class Context:
         _check(self._lib.sp_determine_pattern(self._h, _view(q), _view(k), _i32(heads), len(heads), block,
                                               _ptr(pivot_last_rows), _i32(row_of_head), delta, tau, _ptr(pattern_out),
                                               _ptr(dist_out), _stream(stream)), "sp_determine_pattern")
+
+    def sp_vertical_slash_pattern(self, q, k, heads, gamma, block, mask_out, counts_out, indices_out, sel_v_out=None,
+                                  sel_s_out=None, stream=None):
+        heads = list(heads)
+        _check(self._lib.sp_vertical_slash_pattern(self._h, _view(q), _view(k), _i32(heads), len(heads), gamma, block,
+                                                   _ptr(mask_out), _ptr(counts_out), _ptr(indices_out), _ptr(sel_v_out),
+                                                   _ptr(sel_s_out), _stream(stream)), "sp_vertical_slash_pattern")
 
     def sp_prefill_attn_host(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
         """Host tensors (bf16, contiguous, preferably pinned): q, out [Hq, N, d]; k, v [Hkv, N, d]; mask_out u8 [Hq, Nb, Nb]."""

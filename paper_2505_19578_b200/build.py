@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libshareprefill.so")
-SOURCES = ["api.cu", "attn_pair.cu", "attn_tc.cu", "attn_simt.cu", "mask_kernel.cu", "pooled_pattern.cu"]
+SOURCES = ["api.cu", "attn_pair.cu", "attn_tc.cu", "attn_simt.cu", "mask_kernel.cu", "pooled_pattern.cu", "vslash.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "shareprefill.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

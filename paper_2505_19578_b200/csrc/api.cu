@@ -673,4 +673,39 @@ int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   return SP_OK;
 }
 
+int sp_vertical_slash_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads, int n_heads,
+                              float gamma, int block, uint8_t* mask_out, int32_t* counts_out, int32_t* indices_out,
+                              uint8_t* sel_v_out, uint8_t* sel_s_out, void* stream) {
+  if (!ctx || !heads || n_heads < 0 || !mask_out || !counts_out || !indices_out) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, k, q, block, &p);
+  if (rc) return rc;
+  if (p.d != 128 || p.B != 128) return SP_ERR_UNSUPPORTED;
+  if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  for (int t = 0; t < n_heads; ++t)
+    if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
+  if (n_heads == 0) return SP_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  VslashArgs v;
+  memset(&v, 0, sizeof(v));
+  v.chunk = 8;
+  if ((rc = reserve(ctx, align_up(vslash_scratch_bytes(n_heads, p.N, v.chunk))))) return rc;
+  v.q = static_cast<const __nv_bfloat16*>(q->data);
+  v.k = static_cast<const __nv_bfloat16*>(k->data);
+  v.q_sh = q->stride[1]; v.q_sn = q->stride[2];
+  v.k_sh = k->stride[1]; v.k_sn = k->stride[2];
+  v.n_q_heads = p.Hq; v.n_kv_heads = p.Hkv; v.N = p.N; v.d = p.d; v.B = p.B; v.n_heads = n_heads;
+  for (int t = 0; t < n_heads; ++t) v.heads.v[t] = heads[t];
+  v.gamma = (double)gamma;
+  v.scratch = ctx->ws;
+  v.mask = mask_out; v.counts = counts_out; v.indices = indices_out;
+  v.sel_v_out = sel_v_out; v.sel_s_out = sel_s_out;
+  v.status = ctx->status;
+  if (launch_vertical_slash(v, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  ctx->launches += 8;
+  return SP_OK;
+}
+
 }  // extern "C"

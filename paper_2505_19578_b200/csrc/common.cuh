@@ -63,6 +63,23 @@ struct PooledArgs {
   float* pooled;   // out [n_heads, Nb, Nb]  (launch_determine_pattern: [n_heads, Nb], the last row only)
 };
 
+// Vertical-slash search (Algorithm "Search Vertical Slash Pattern").  Strides in elements.
+struct VslashArgs {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  int64_t q_sh, q_sn, k_sh, k_sn;
+  int n_q_heads, n_kv_heads, N, d, B, n_heads, chunk;
+  HeadTable heads;
+  double gamma;
+  void* scratch;            // vslash_scratch_bytes(n_heads, N, chunk)
+  uint8_t* mask;            // out [n_heads, Nb, Nb]
+  int32_t* counts;          // out [n_heads, Nb]
+  int32_t* indices;         // out [n_heads, Nb, Nb]
+  uint8_t* sel_v_out;       // optional out [n_heads, N]: selected key columns
+  uint8_t* sel_s_out;       // optional out [n_heads, N]: selected query-minus-key offsets
+  int* status;
+};
+
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TMEM / TMA, one row-block per CTA
@@ -79,6 +96,9 @@ cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s);
 cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
                                        uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
                                        cudaStream_t s);
+cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s);
+size_t vslash_scratch_bytes(int n_heads, int N, int chunk);
+cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s);
 cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,
                                      float delta, float tau, int32_t* pattern, float* dist, cudaStream_t s);
 

@@ -392,6 +392,13 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
   return cudaGetLastError();
 }
 
+cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s) {
+  const long rows = (long)n_maps * nb;
+  if (rows == 0) return cudaSuccess;
+  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,
                                      float delta, float tau, int32_t* pattern, float* dist, cudaStream_t s) {
   if (a.n_heads == 0) return cudaSuccess;

@@ -153,3 +153,73 @@ def test_determine_pattern_matches_oracle(binding, name, seq):
     for t, p in enumerate(piv):
         if rows[p] == t:
             assert got_d[p, 1] <= 2e-3
+
+
+# ------------------------------------------------------------------ vertical-slash search
+
+VS_BAND = 2e-5         # a line may flip only if the oracle's cumulative score at it is this close to gamma
+
+
+def _cum_at(a, g):
+    f = a / a.sum()
+    order = np.argsort(-f, kind="stable")
+    cum = np.empty(len(a))
+    cum[order] = np.cumsum(f[order])
+    return cum, f
+
+
+@pytest.mark.parametrize("name,seq,gamma", [("llama8b_32k", 4096, 0.9), ("qwen7b_64k", 2048, 0.8), ("llama8b_128k", 8192, 0.95)])
+def test_vertical_slash_pattern_matches_oracle(binding, name, seq, gamma):
+    from oracle import shareprefill_oracle as orc
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=6)
+    cfg = L["cfg"]
+    B, Nb, N = cfg.block, cfg.seq // cfg.block, cfg.seq
+    heads = [1, cfg.n_q_heads - 1, 0]
+    ctx = binding.Context()
+    q, k, v = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+    mask = torch.full((len(heads), Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+    counts = torch.full((len(heads), Nb), -5, dtype=torch.int32, device="cuda")
+    idx = torch.full((len(heads), Nb, Nb), -5, dtype=torch.int32, device="cuda")
+    sv = torch.full((len(heads), N), 9, dtype=torch.uint8, device="cuda")
+    ss = torch.full((len(heads), N), 9, dtype=torch.uint8, device="cuda")
+    for rep in range(2):                                       # the second call reuses the scratch counters
+        ctx.sp_vertical_slash_pattern(q, k, heads, gamma, B, mask, counts, idx, sel_v_out=sv, sel_s_out=ss)
+        torch.cuda.synchronize()
+        assert ctx.status() == (0, 0)
+    Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
+    g = par.gamma32(gamma)
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    for t, h in enumerate(heads):
+        res = ppo.search_vertical_slash_pattern(Q[h], K[h // G], g, B)
+        for got, want, a in ((sv[t].cpu().numpy(), res["sel_v"], res["a_v"]), (ss[t].cpu().numpy(), res["sel_s"], res["a_s"])):
+            cum, f = _cum_at(a, g)
+            diff = np.flatnonzero(got.astype(bool) != want)
+            for e in diff:
+                assert abs(cum[e] - g) <= VS_BAND or abs(cum[e] - f[e] - g) <= VS_BAND, (h, e, cum[e], g)
+            assert len(diff) <= 4
+        m = mask[t].cpu().numpy()
+        # the mask is exactly what the GPU's own selected lines imply (integer work: bit-exact)
+        gv, gs = sv[t].cpu().numpy().astype(bool), ss[t].cpu().numpy().astype(bool)
+        want = np.zeros((Nb, Nb), np.uint8)
+        colb = gv.reshape(Nb, B).any(axis=1)
+        for i in range(Nb):
+            for j in range(i + 1):
+                lo, hi = max((i - j) * B - (B - 1), 0), min((i - j) * B + (B - 1), N - 1)
+                want[i, j] = colb[j] or gs[lo:hi + 1].any()
+            if want[i].sum() == 0:
+                want[i, i] = 1
+        assert np.array_equal(m, want)
+        if np.array_equal(gv, res["sel_v"]) and np.array_equal(gs, res["sel_s"]):
+            assert np.array_equal(m, res["mask"])
+        c, ix = counts[t].cpu().numpy(), idx[t].cpu().numpy()
+        for i in range(Nb):
+            sel = np.flatnonzero(m[i])
+            assert c[i] == len(sel) and np.array_equal(ix[i, :c[i]], sel) and np.all(ix[i, c[i]:] == -1)
+    # the lists drive the block-sparse kernel directly
+    out = torch.full_like(q, float("nan"))
+    ctx.sp_block_sparse_attn(q, k, v, heads, list(range(len(heads))), counts, idx, B, out)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    for t, h in enumerate(heads[:2]):
+        ref = orc.masked_attention(Q, K, V, h, mask[t].cpu().numpy(), B)
+        par.assert_out_close(par.f64(out[h]), ref, f"head {h}")
