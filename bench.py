@@ -319,6 +319,24 @@ def run_ours(args):
         torch.cuda.synchronize()
         literal_step(le)
         torch.cuda.synchronize()
+        # vertical-slash fallback of every member head: search, then the block-sparse kernel on its lists
+        vs = None
+        if (cfg.head_dim, B) == (128, 128):
+            vm = torch.empty(len(members), Nb, Nb, dtype=torch.uint8, device=dev)
+            vc = torch.empty(len(members), Nb, dtype=torch.int32, device=dev)
+            vi = torch.empty(len(members), Nb, Nb, dtype=torch.int32, device=dev)
+            ve = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            for _ in range(2):
+                ve[0].record(stream)
+                ctx.sp_vertical_slash_pattern(q, k, members, gamma, B, vm, vc, vi, stream=stream)
+                ve[1].record(stream)
+                ctx.sp_block_sparse_attn(q, k, v, members, list(range(len(members))), vc, vi, B, out, stream=stream)
+                ve[2].record(stream)
+                torch.cuda.synchronize()
+            vtiles = int(vc.sum().item())
+            vs = {"search_ms": ve[0].elapsed_time(ve[1]), "block_sparse_attn_ms": ve[1].elapsed_time(ve[2]),
+                  "heads": len(members), "mean_mask_density": vtiles / (len(members) * tiles_causal),
+                  "block_sparse_tflops": vtiles * tile_flops(cfg) / (ve[1].elapsed_time(ve[2]) * 1e-3) / 1e12}
         inter = (lm & pm).sum(dim=(1, 2)).float()
         union = (lm | pm).sum(dim=(1, 2)).float()
         literal = {
@@ -327,6 +345,7 @@ def run_ours(args):
             "mask_density_per_pivot": {int(p): float(lc[t].sum().item()) / tiles_causal for t, p in enumerate(piv)},
             "jaccard_with_mass_mask_per_pivot": {int(p): float(inter[t] / union[t]) for t, p in enumerate(piv)},
             "heads_shared_pivot_at_delta0.3_tau0.2": int((pat == 0).sum().item()),
+            "vertical_slash": vs,
         }
 
     # ---- end to end through the C ABI with host buffers: H2D of q,k,v, the layer, D2H of the output
