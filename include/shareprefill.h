@@ -302,6 +302,32 @@ int sp_vertical_slash_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* 
                               int n_heads, float gamma, int block, uint8_t* mask_out, int32_t* counts_out,
                               int32_t* indices_out, uint8_t* sel_v_out, uint8_t* sel_s_out, void* stream);
 
+/*
+ * sp_prefill_attn_auto - one layer of Algorithm "Sparse Attention" with the
+ *   pattern decision made on the device, no host synchronisation:
+ *     1. the listed pivot heads (heads whose cluster has no pivotal pattern yet)
+ *        run dense and construct their pattern (Algorithm "Construct Pivotal
+ *        Pattern": pooled_construction = 0: true softmax mass cut per row-block,
+ *        as sp_prefill_attn does; 1: the paper-literal block-averaged QK values
+ *        with one global cut, as sp_pattern_from_pooled does);
+ *     2. every other head that has a pivot in its cluster is classified by
+ *        Algorithm "Determine Sparse Pattern" (d_sparse < delta and d_sim < tau:
+ *        it shares the pivot's pattern; otherwise it searches its own
+ *        vertical-slash pattern, Algorithm "Search Vertical Slash Pattern");
+ *     3. those heads run block-sparse attention over the list chosen for them;
+ *        a head whose cluster has no pivot (or id < 0) runs dense.
+ *   head_dim 128 and block 128 only.
+ *     pattern_out  device i32 [n_q_heads] or NULL: 0 dense, 1 shared pivot,
+ *                  2 vertical-slash.
+ *     mask_out     device u8 [n_q_heads, Nb, Nb] or NULL: the pattern each head
+ *                  used (a pivot: the pattern it constructed).
+ *   Other arguments as for sp_prefill_attn.
+ */
+int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                         const int32_t* cluster_map, const int32_t* pivot_heads, int n_pivots,
+                         float gamma, float delta, float tau, int block, int pooled_construction,
+                         sp_tensor* out, uint8_t* mask_out, int32_t* pattern_out, void* stream);
+
 /* Which attention kernel the context launches: 0 = tensor-core kernels
  * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V

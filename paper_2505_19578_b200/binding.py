@@ -30,7 +30,7 @@ EXPORTS = (
     "sp_strerror", "sp_dense_pivot_attn", "sp_block_mask_from_importance", "sp_block_sparse_attn",
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
-    "sp_determine_pattern", "sp_vertical_slash_pattern",
+    "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
 )
 
 
@@ -77,6 +77,7 @@ def load() -> ctypes.CDLL:
     lib.sp_pattern_from_pooled.argtypes = [P, P, I, I, F, P, P, P, P, P]
     lib.sp_determine_pattern.argtypes = [P, T, T, IP, I, I, P, IP, F, F, P, P, P]
     lib.sp_vertical_slash_pattern.argtypes = [P, T, T, IP, I, F, I, P, P, P, P, P, P]
+    lib.sp_prefill_attn_auto.argtypes = [P, T, T, T, IP, IP, I, F, F, F, I, I, T, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
@@ -216,6 +217,14 @@ class Context:
         _check(self._lib.sp_vertical_slash_pattern(self._h, _view(q), _view(k), _i32(heads), len(heads), gamma, block,
                                                    _ptr(mask_out), _ptr(counts_out), _ptr(indices_out), _ptr(sel_v_out),
                                                    _ptr(sel_s_out), _stream(stream)), "sp_vertical_slash_pattern")
+
+    def sp_prefill_attn_auto(self, q, k, v, cluster_map, pivot_heads, gamma, delta, tau, block, out, pooled_construction=False,
+                             mask_out=None, pattern_out=None, stream=None):
+        cluster_map, pivot_heads = list(cluster_map), list(pivot_heads)
+        _check(self._lib.sp_prefill_attn_auto(self._h, _view(q), _view(k), _view(v), _i32(cluster_map), _i32(pivot_heads),
+                                              len(pivot_heads), gamma, delta, tau, block, int(bool(pooled_construction)),
+                                              _view(out), _ptr(mask_out), _ptr(pattern_out), _stream(stream)),
+               "sp_prefill_attn_auto")
 
     def sp_prefill_attn_host(self, q, k, v, cluster_map, pivot_heads, gamma, block, out, mask_out=None, stream=None):
         """Host tensors (bf16, contiguous, preferably pinned): q, out [Hq, N, d]; k, v [Hkv, N, d]; mask_out u8 [Hq, Nb, Nb]."""

@@ -152,9 +152,9 @@ WsLayout ws_layout(int Nb, int B, int n_pivots) {
 }
 
 __global__ void gather_masks_kernel(const uint8_t* __restrict__ pivot_masks, HeadTable src, int nb,
-                                    uint8_t* __restrict__ out) {
+                                    uint8_t* __restrict__ out, const int32_t* __restrict__ src_dev = nullptr) {
   const int i = blockIdx.x, h = blockIdx.y;
-  const int s = src.v[h];
+  const int s = src_dev ? src_dev[h] : src.v[h];
   uint8_t* dst = out + ((size_t)h * nb + i) * nb;
   if (s >= 0) {
     const uint8_t* from = pivot_masks + ((size_t)s * nb + i) * nb;
@@ -705,6 +705,161 @@ int sp_vertical_slash_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* 
   v.status = ctx->status;
   if (launch_vertical_slash(v, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
   ctx->launches += 8;
+  return SP_OK;
+}
+
+int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v, const int32_t* cluster_map,
+                         const int32_t* pivot_heads, int n_pivots, float gamma, float delta, float tau, int block,
+                         int pooled_construction, sp_tensor* out, uint8_t* mask_out, int32_t* pattern_out, void* stream) {
+  if (!ctx || !cluster_map || n_pivots < 0 || (n_pivots > 0 && !pivot_heads)) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (p.d != 128 || p.B != 128) return SP_ERR_UNSUPPORTED;       // the vertical-slash search
+  if (n_pivots > p.Hq) return SP_ERR_INVALID_ARG;
+  int pivot_slot_of_head[kMaxHeads];
+  HeadTable piv_heads;
+  for (int h = 0; h < p.Hq; ++h) pivot_slot_of_head[h] = -1;
+  for (int t = 0; t < n_pivots; ++t) {
+    const int h = pivot_heads[t];
+    if (h < 0 || h >= p.Hq || pivot_slot_of_head[h] >= 0) return SP_ERR_INVALID_ARG;
+    pivot_slot_of_head[h] = t;
+    piv_heads.v[t] = h;
+  }
+  auto cluster_pivot = [&](int c) {
+    if (c < 0) return -1;
+    for (int t = 0; t < n_pivots; ++t)
+      if (cluster_map[pivot_heads[t]] == c) return t;
+    return -1;
+  };
+  HeadTable member_heads, member_pivot;
+  int member_list[kMaxHeads];
+  int n_members = 0;
+  for (int h = 0; h < p.Hq; ++h) {
+    if (pivot_slot_of_head[h] >= 0) continue;
+    member_heads.v[n_members] = h;
+    member_pivot.v[n_members] = cluster_pivot(cluster_map[h]);
+    member_list[n_members] = h;
+    ++n_members;
+  }
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // workspace
+  const size_t nn = (size_t)p.Nb * p.Nb;
+  const int n_lists = n_pivots + n_members;
+  const int n_row = n_pivots > n_members ? n_pivots : n_members;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  const size_t o_imp = take(n_pivots * nn * sizeof(float));
+  const size_t o_scores = take(pooled_construction ? n_pivots * nn * sizeof(float) : 0);
+  const size_t o_mask = take(n_lists * nn);
+  const size_t o_counts = take((size_t)n_lists * p.Nb * sizeof(int32_t));
+  const size_t o_indices = take(n_lists * nn * sizeof(int32_t));
+  const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_pivots, p.Nb, p.d) * sizeof(float)
+                                                    : (size_t)n_pivots * tile_stats_bytes_per_head(p.Nb, p.B));
+  const size_t o_atilde = take((size_t)n_pivots * p.Nb * sizeof(float));
+  const size_t o_rows = take((size_t)n_row * p.Nb * sizeof(float));
+  const size_t o_small = take((size_t)(3 * kMaxHeads + p.Hq) * sizeof(int32_t));
+  const size_t o_vs = take(vslash_scratch_bytes(n_members, p.N, 8));
+  if ((rc = reserve(ctx, off))) return rc;
+  char* ws = static_cast<char*>(ctx->ws);
+  float* imp = reinterpret_cast<float*>(ws + o_imp);
+  uint8_t* masks = reinterpret_cast<uint8_t*>(ws + o_mask);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + o_counts);
+  int32_t* indices = reinterpret_cast<int32_t*>(ws + o_indices);
+  float* a_tilde = reinterpret_cast<float*>(ws + o_atilde);
+  float* rows_scratch = reinterpret_cast<float*>(ws + o_rows);
+  int32_t* decide = reinterpret_cast<int32_t*>(ws + o_small);
+  int32_t* lists_dev = decide + kMaxHeads;
+  int32_t* active = lists_dev + kMaxHeads;
+  int32_t* src_dev = active + kMaxHeads;
+
+  // 1. heads without a pivotal pattern: dense attention (Algorithm "Share Pivotal Pattern": all-ones pattern)
+  AttnArgs a = base_args(ctx, p, q, k, v, out);
+  a.n_heads = n_pivots;
+  for (int t = 0; t < n_pivots; ++t) { a.heads.v[t] = pivot_heads[t]; a.lists.v[t] = -1; }
+  if (!pooled_construction) {
+    a.importance = imp;
+    a.tile_stats = reinterpret_cast<float*>(ws + o_scratch);
+  }
+  if ((rc = launch_attn(ctx, a, s))) return rc;
+
+  // 2. Algorithm "Construct Pivotal Pattern": lists of the pivots in slots 0..n_pivots-1, and their representatives a~
+  if (n_pivots > 0) {
+    if (pooled_construction) {
+      PooledArgs pa = pooled_args(p, q, k, pivot_heads, n_pivots);
+      pa.qbar = reinterpret_cast<float*>(ws + o_scratch);
+      pa.kbar = pa.qbar + (size_t)n_pivots * p.Nb * p.d;
+      pa.diag = pa.kbar + (size_t)n_pivots * p.Nb * p.d;
+      pa.pooled = imp;
+      if (launch_pooled_logits(pa, s) != cudaSuccess) return SP_ERR_CUDA;
+      if (launch_pattern_from_pooled(imp, n_pivots, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores), masks, counts,
+                                     indices, nullptr, s) != cudaSuccess)
+        return SP_ERR_CUDA;
+      ctx->launches += 5;
+    } else {
+      MaskArgs m{imp, n_pivots, p.Nb, (double)gamma, masks, counts, indices};
+      if (launch_block_mask(m, s) != cudaSuccess) return SP_ERR_CUDA;
+      ctx->launches += 1;
+    }
+    PooledArgs pl = pooled_args(p, q, k, pivot_heads, n_pivots);
+    pl.pooled = rows_scratch;
+    if (launch_last_row_distribution(pl, a_tilde, s) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 2;
+  }
+
+  // 3. Algorithm "Determine Sparse Pattern" for every other head, on the device
+  if (n_members > 0) {
+    PooledArgs pm = pooled_args(p, q, k, member_list, n_members);
+    pm.pooled = rows_scratch;
+    if (launch_determine_pattern(pm, a_tilde, member_pivot, delta, tau, decide, nullptr, s) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 2;
+  }
+  if (launch_finalize_pattern(decide, member_pivot, member_heads, n_members, piv_heads, n_pivots, lists_dev, active, pattern_out,
+                              src_dev, s) != cudaSuccess)
+    return SP_ERR_CUDA;
+  ctx->launches += 1;
+
+  // 4. Algorithm "Search Vertical Slash Pattern" for the heads that do not share: lists in slots n_pivots + member
+  if (n_members > 0) {
+    VslashArgs vs;
+    memset(&vs, 0, sizeof(vs));
+    vs.chunk = 8;
+    vs.q = static_cast<const __nv_bfloat16*>(q->data);
+    vs.k = static_cast<const __nv_bfloat16*>(k->data);
+    vs.q_sh = q->stride[1]; vs.q_sn = q->stride[2];
+    vs.k_sh = k->stride[1]; vs.k_sn = k->stride[2];
+    vs.n_q_heads = p.Hq; vs.n_kv_heads = p.Hkv; vs.N = p.N; vs.d = p.d; vs.B = p.B; vs.n_heads = n_members;
+    vs.heads = member_heads;
+    vs.gamma = (double)gamma;
+    vs.scratch = ws + o_vs;
+    vs.mask = masks + (size_t)n_pivots * nn;
+    vs.counts = counts + (size_t)n_pivots * p.Nb;
+    vs.indices = indices + (size_t)n_pivots * nn;
+    vs.active = active;
+    vs.status = ctx->status;
+    if (launch_vertical_slash(vs, s) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 8;
+
+    // 5. sparse attention of those heads over the list chosen for each
+    AttnArgs b = base_args(ctx, p, q, k, v, out);
+    b.counts = counts;
+    b.indices = indices;
+    b.n_heads = n_members;
+    for (int t = 0; t < n_members; ++t) { b.heads.v[t] = member_heads.v[t]; b.lists.v[t] = -1; }
+    b.lists_dev = lists_dev;
+    if ((rc = launch_attn(ctx, b, s))) return rc;
+  }
+  if (mask_out) {
+    HeadTable unused;
+    memset(&unused, 0, sizeof(unused));
+    gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, s>>>(masks, unused, p.Nb, mask_out, src_dev);
+    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+  }
   return SP_OK;
 }
 

@@ -178,7 +178,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   const int slot = blockIdx.x;
   const int h = a.heads.v[slot];
   const int g = h / a.group;
-  const int list = a.lists.v[slot];
+  const int list = a.lists_dev ? a.lists_dev[slot] : a.lists.v[slot];   // decided on the device, or by the host
   const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
   TileInfo tile[2];
 #pragma unroll

@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_simt_kernel(const AttnArgs a
   const int slot = blockIdx.y;
   const int h = a.heads.v[slot];
   const int g = h / a.group;
-  const int list = a.lists.v[slot];
+  const int list = a.lists_dev ? a.lists_dev[slot] : a.lists.v[slot];   // decided on the device, or by the host
   const int B = a.B;
   const int cnt = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
   const int32_t* idx = list >= 0 ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;

@@ -82,7 +82,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
   const int slot = blockIdx.y;
   const int h = a.heads.v[slot];
   const int g = h / a.group;
-  const int list = a.lists.v[slot];
+  const int list = a.lists_dev ? a.lists_dev[slot] : a.lists.v[slot];   // decided on the device, or by the host
   int cnt = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
   cnt = cnt < 0 ? 0 : (cnt > i + 1 ? i + 1 : cnt);
   const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work

@@ -29,6 +29,7 @@ struct AttnArgs {
   int n_heads;             // heads processed by this launch
   HeadTable heads;         // query-head index per slot
   HeadTable lists;         // list index per slot, -1 = dense (all causal tiles)
+  const int32_t* lists_dev;  // if not null: list index per slot read from device memory instead
   const int32_t* counts;   // [n_lists, Nb]       (may be null when every slot is dense)
   const int32_t* indices;  // [n_lists, Nb, Nb]
   float* importance;       // [n_heads, Nb, Nb] or null
@@ -77,6 +78,7 @@ struct VslashArgs {
   int32_t* indices;         // out [n_heads, Nb, Nb]
   uint8_t* sel_v_out;       // optional out [n_heads, N]: selected key columns
   uint8_t* sel_s_out;       // optional out [n_heads, N]: selected query-minus-key offsets
+  const int32_t* active;    // optional device [n_heads]: heads with 0 are skipped (their outputs are undefined)
   int* status;
 };
 
@@ -96,11 +98,16 @@ cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s);
 cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
                                        uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
                                        cudaStream_t s);
+cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivot_slot_of_member, const HeadTable& head_of_member,
+                                    int n_members, const HeadTable& pivot_heads, int n_pivots, int32_t* lists_dev,
+                                    int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s);
 cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s);
 size_t vslash_scratch_bytes(int n_heads, int N, int chunk);
 cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s);
 cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,
                                      float delta, float tau, int32_t* pattern, float* dist, cudaStream_t s);
+// softmax of the pooled last row of each listed head (the representative a~ / a^): out [n_heads, Nb]; a.pooled is scratch [n_heads, Nb]
+cudaError_t launch_last_row_distribution(const PooledArgs& a, float* out, cudaStream_t s);
 
 // bytes of per-tile softmax statistics the tensor-core kernel spills for one head
 inline size_t tile_stats_bytes_per_head(int Nb, int B) {

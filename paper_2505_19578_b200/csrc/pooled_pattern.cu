@@ -392,6 +392,79 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
   return cudaGetLastError();
 }
 
+namespace {
+
+// softmax of each row of z [n, nb] -> out; one CTA of 256 threads per row
+__global__ void row_softmax_kernel(const float* __restrict__ z, int nb, float* __restrict__ out) {
+  __shared__ float red[8];
+  __shared__ float bc;
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* in = z + (size_t)row * nb;
+  float m = -CUDART_INF_F;
+  for (int j = tid; j < nb; j += blockDim.x) m = fmaxf(m, in[j]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  if (tid == 0) { float t = red[0]; for (int w = 1; w < 8; ++w) t = fmaxf(t, red[w]); bc = t; }
+  __syncthreads();
+  m = bc;
+  float s = 0.f;
+  for (int j = tid; j < nb; j += blockDim.x) s += expf(in[j] - m);
+  s = warp_sum(s);
+  __syncthreads();
+  if (lane == 0) red[warp] = s;
+  __syncthreads();
+  if (tid == 0) { float t = 0.f; for (int w = 0; w < 8; ++w) t += red[w]; bc = t; }
+  __syncthreads();
+  const float inv = 1.f / bc;
+  for (int j = tid; j < nb; j += blockDim.x) out[(size_t)row * nb + j] = expf(in[j] - m) * inv;
+}
+
+}  // namespace
+
+cudaError_t launch_last_row_distribution(const PooledArgs& a, float* out, cudaStream_t s) {
+  if (a.n_heads == 0) return cudaSuccess;
+  last_row_pooled_kernel<<<dim3(a.Nb, a.n_heads), a.d, 0, s>>>(a);
+  row_softmax_kernel<<<a.n_heads, 256, 0, s>>>(a.pooled, a.Nb, out);
+  return cudaGetLastError();
+}
+
+namespace {
+// decisions of "Determine Sparse Pattern" -> which list each member walks, which members need the
+// vertical-slash search, pattern codes (0 dense, 1 shared pivot, 2 vertical-slash) and mask sources per head
+__global__ void finalize_pattern_kernel(const int32_t* __restrict__ decide, HeadTable pivot_slot_of_member,
+                                        HeadTable head_of_member, int n_members, HeadTable pivot_heads, int n_pivots,
+                                        int32_t* __restrict__ lists_dev, int32_t* __restrict__ active,
+                                        int32_t* __restrict__ pattern_out, int32_t* __restrict__ src_dev) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n_members) {
+    const int ps = pivot_slot_of_member.v[t], h = head_of_member.v[t];
+    int list, act, code;
+    if (ps < 0) { list = -1; act = 0; code = 0; }                       // no pivotal pattern for its cluster: dense
+    else if (decide[t] == 0) { list = ps; act = 0; code = 1; }          // shares the pivot's pattern
+    else { list = n_pivots + t; act = 1; code = 2; }                    // falls back to its own vertical-slash pattern
+    lists_dev[t] = list;
+    active[t] = act;
+    src_dev[h] = list;
+    if (pattern_out) pattern_out[h] = code;
+  } else if (t < n_members + n_pivots) {
+    const int p = t - n_members, h = pivot_heads.v[p];
+    src_dev[h] = p;
+    if (pattern_out) pattern_out[h] = 0;
+  }
+}
+}  // namespace
+
+cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivot_slot_of_member, const HeadTable& head_of_member,
+                                    int n_members, const HeadTable& pivot_heads, int n_pivots, int32_t* lists_dev,
+                                    int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s) {
+  const int n = n_members + n_pivots;
+  if (n == 0) return cudaSuccess;
+  finalize_pattern_kernel<<<(n + 127) / 128, 128, 0, s>>>(decide, pivot_slot_of_member, head_of_member, n_members, pivot_heads,
+                                                          n_pivots, lists_dev, active, pattern_out, src_dev);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s) {
   const long rows = (long)n_maps * nb;
   if (rows == 0) return cudaSuccess;

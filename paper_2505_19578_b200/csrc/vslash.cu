@@ -54,6 +54,7 @@ struct VsArgs {
   float* lse2;                   // [n_heads, 128]
   float* a_v;                    // [n_heads, N]
   unsigned long long* a_s_fx;    // [n_heads, N], 2^-40 fixed point
+  const int32_t* active;
   int* status;
 };
 
@@ -76,6 +77,7 @@ vs_sweep_kernel(const VsArgs a, const __grid_constant__ CUtensorMap tm_q, const 
   const int j0 = chunk * a.chunk;
   int n_tiles = a.Nb - j0 < a.chunk ? a.Nb - j0 : a.chunk;
   if (*reinterpret_cast<volatile int*>(a.status) != 0) n_tiles = 0;     // an earlier wait ran out: do no work
+  if (a.active && a.active[slot] == 0) n_tiles = 0;                      // head not selected for the search
   const int last = a.Nb - 1;
   const Abort ab{abort_flag, a.status};
 
@@ -267,7 +269,8 @@ struct VSel {
 
 // grid = n_vectors; vector v at scores + v * n
 __global__ void __launch_bounds__(kSelThreads) vector_select_kernel(const float* __restrict__ scores, long n, double gamma,
-                                                                    uint8_t* __restrict__ sel) {
+                                                                    uint8_t* __restrict__ sel, const int32_t* __restrict__ active) {
+  if (active && active[blockIdx.x] == 0) return;
   extern __shared__ unsigned char vsel_raw[];
   VSel& sh = *reinterpret_cast<VSel*>(vsel_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -412,6 +415,7 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   a.N = v.N; a.Nb = Nb; a.n_heads = v.n_heads; a.chunk = chunk; a.heads = v.heads;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
   a.status = v.status;
+  a.active = v.active;
   CUtensorMap tq, tk;
   if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
       !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK))
@@ -427,8 +431,8 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   const long n_all = (long)v.n_heads * v.N;
   vs_slash_to_float_kernel<<<(unsigned)((n_all + 255) / 256), 256, 0, s>>>(a.a_s_fx, n_all, a_s);
   // a_v and a_s are adjacent: 2 * n_heads vectors of N scores (up() keeps them adjacent when n_heads * N * 4 is a multiple of 256)
-  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a.a_v, v.N, v.gamma, sel);
-  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N);
+  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a.a_v, v.N, v.gamma, sel, v.active);
+  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
   vs_lines_to_mask_kernel<<<v.n_heads, 512, 0, s>>>(sel, sel + (size_t)v.n_heads * v.N, v.N, Nb, v.mask);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if (v.sel_v_out) {

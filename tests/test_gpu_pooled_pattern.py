@@ -223,3 +223,104 @@ def test_vertical_slash_pattern_matches_oracle(binding, name, seq, gamma):
     for t, h in enumerate(heads[:2]):
         ref = orc.masked_attention(Q, K, V, h, mask[t].cpu().numpy(), B)
         par.assert_out_close(par.f64(out[h]), ref, f"head {h}")
+
+
+# ------------------------------------------------------------------ the whole decision flow on the device
+
+@pytest.mark.parametrize("pooled", [False, True])
+@pytest.mark.parametrize("name,seq", [("llama8b_32k", 4096), ("qwen7b_64k", 2048)])
+def test_prefill_attn_auto_is_the_composition_of_its_steps(binding, name, seq, pooled):
+    """sp_prefill_attn_auto must equal what the separately tested calls give when chained by hand with the
+    decisions read back, and its outputs must match the oracle's masked attention under the masks it reports."""
+    from oracle import shareprefill_oracle as orc
+    L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=8)
+    cfg = L["cfg"]
+    B, Nb, Hq = cfg.block, cfg.seq // cfg.block, cfg.n_q_heads
+    cm = list(L["cluster_map"])
+    piv = list(L["pivot_heads"])
+    cm[-1] = -1                                               # one head without a cluster: dense
+    if Hq - 1 in piv:
+        piv.remove(Hq - 1)
+    gamma = 0.9
+    ctx = binding.Context()
+    q, k, v = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+    members = [h for h in range(Hq) if h not in piv]
+    first = {}
+    for t, p in enumerate(piv):
+        first.setdefault(cm[p], t)
+    rows = [first.get(cm[h], -1) if cm[h] >= 0 else -1 for h in members]
+
+    # --- by hand: pivots' representatives, distances of the members, thresholds that split them
+    Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
+    G = Hq // cfg.n_kv_heads
+    a_t = [ppo.last_block_distribution(Q[p], K[p // G], B) for p in piv]
+    ref = [ppo.determine_pattern(ppo.last_block_distribution(Q[h], K[h // G], B), a_t[r] if r >= 0 else None, 1.0, 1.0)
+           for h, r in zip(members, rows)]
+    ds = sorted(r[1] for r, row in zip(ref, rows) if row >= 0)
+    delta = ds[len(ds) // 2] + 1e-3 if ds[-1] - ds[0] > 5e-3 else ds[-1] + 1.0
+    dm = sorted(r[2] for r, row in zip(ref, rows) if row >= 0)
+    tau = dm[(2 * len(dm)) // 3] + 1e-3
+
+    out = torch.full_like(q, float("nan"))
+    mask = torch.full((Hq, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+    pat = torch.full((Hq,), -1, dtype=torch.int32, device="cuda")
+    ctx.sp_prefill_attn_auto(q, k, v, cm, piv, gamma, delta, tau, B, out, pooled_construction=pooled, mask_out=mask,
+                             pattern_out=pat)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    pat_h, mask_h = pat.cpu().numpy(), mask.cpu().numpy()
+
+    # decisions: as the oracle's wherever the distances are clear of the thresholds
+    kinds = set()
+    for h, r, (_, d1, d2) in zip(members, rows, ref):
+        if r < 0:
+            assert pat_h[h] == 0
+            continue
+        want = 1 if (d1 < delta and d2 < tau) else 2
+        if min(abs(d1 - delta), abs(d2 - tau)) > DIST_MARGIN:
+            assert pat_h[h] == want, (h, d1, d2, delta, tau)
+        kinds.add(int(pat_h[h]))
+    assert all(pat_h[p] == 0 for p in piv)
+    assert kinds == {1, 2}                                    # both branches are exercised
+
+    # masks: pivots' as the construction call gives them, members' by their decision
+    if pooled:
+        pl = torch.empty(len(piv), Nb, Nb, device="cuda")
+        ctx.sp_pooled_logits(q, k, piv, B, pl)
+        pmask = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device="cuda")
+        pc = torch.empty(len(piv), Nb, dtype=torch.int32, device="cuda")
+        pi = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device="cuda")
+        ctx.sp_pattern_from_pooled(pl, gamma, pmask, pc, pi)
+    else:
+        imp = torch.empty(len(piv), Nb, Nb, device="cuda")
+        tmp = torch.empty_like(q)
+        ctx.sp_dense_pivot_attn(q, k, v, piv, B, tmp, importance_out=imp)
+        pmask = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device="cuda")
+        pc = torch.empty(len(piv), Nb, dtype=torch.int32, device="cuda")
+        pi = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device="cuda")
+        ctx.sp_block_mask_from_importance(imp, gamma, pmask, pc, pi)
+    vs_heads = [h for h in members if pat_h[h] == 2]
+    vmask = torch.empty(len(vs_heads), Nb, Nb, dtype=torch.uint8, device="cuda")
+    vc = torch.empty(len(vs_heads), Nb, dtype=torch.int32, device="cuda")
+    vi = torch.empty(len(vs_heads), Nb, Nb, dtype=torch.int32, device="cuda")
+    ctx.sp_vertical_slash_pattern(q, k, vs_heads, gamma, B, vmask, vc, vi)
+    torch.cuda.synchronize()
+    pmask_h, vmask_h = pmask.cpu().numpy(), vmask.cpu().numpy()
+    tri = np.tril(np.ones((Nb, Nb), np.uint8))
+    for t, p in enumerate(piv):
+        assert np.array_equal(mask_h[p], pmask_h[t])
+    for h, r in zip(members, rows):
+        if pat_h[h] == 0:
+            assert np.array_equal(mask_h[h], tri)
+        elif pat_h[h] == 1:
+            assert np.array_equal(mask_h[h], pmask_h[r])
+        else:
+            assert np.array_equal(mask_h[h], vmask_h[vs_heads.index(h)])
+
+    # outputs: dense for pivots and unclustered heads, masked attention under the reported mask for the rest
+    check = piv[:1] + [Hq - 1] + [h for h in members if pat_h[h] == 1][:1] + vs_heads[:1]
+    for h in check:
+        M = tri if pat_h[h] == 0 else mask_h[h]
+        refo = orc.masked_attention(Q, K, V, h, M, B)
+        par.assert_out_close(par.f64(out[h]), refo, f"head {h} (pattern {pat_h[h]})")
+    assert torch.isfinite(out.float()).all()
