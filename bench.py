@@ -337,6 +337,20 @@ def run_ours(args):
             vs = {"search_ms": ve[0].elapsed_time(ve[1]), "block_sparse_attn_ms": ve[1].elapsed_time(ve[2]),
                   "heads": len(members), "mean_mask_density": vtiles / (len(members) * tiles_causal),
                   "block_sparse_tflops": vtiles * tile_flops(cfg) / (ve[1].elapsed_time(ve[2]) * 1e-3) / 1e12}
+        # the whole online algorithm with the decision on the device (paper's thresholds, then thresholds that let heads share)
+        auto = None
+        if (cfg.head_dim, B) == (128, 128):
+            auto = {}
+            for label, (dl, tu) in (("delta0.3_tau0.2", (0.3, 0.2)), ("delta1_tau1", (1.0, 1.0))):
+                ae = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                for _ in range(2):
+                    ae[0].record(stream)
+                    ctx.sp_prefill_attn_auto(q, k, v, cm, piv, gamma, dl, tu, B, out, pattern_out=pat, stream=stream)
+                    ae[1].record(stream)
+                    torch.cuda.synchronize()
+                pc_ = pat.cpu().numpy()
+                auto[label] = {"ms_per_layer": ae[0].elapsed_time(ae[1]),
+                               "heads_dense_shared_vslash": [int((pc_ == c).sum()) for c in (0, 1, 2)]}
         inter = (lm & pm).sum(dim=(1, 2)).float()
         union = (lm | pm).sum(dim=(1, 2)).float()
         literal = {
@@ -346,6 +360,7 @@ def run_ours(args):
             "jaccard_with_mass_mask_per_pivot": {int(p): float(inter[t] / union[t]) for t, p in enumerate(piv)},
             "heads_shared_pivot_at_delta0.3_tau0.2": int((pat == 0).sum().item()),
             "vertical_slash": vs,
+            "prefill_attn_auto": auto,
         }
 
     # ---- end to end through the C ABI with host buffers: H2D of q,k,v, the layer, D2H of the output

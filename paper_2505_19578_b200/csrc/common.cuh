@@ -101,7 +101,8 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
 cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivot_slot_of_member, const HeadTable& head_of_member,
                                     int n_members, const HeadTable& pivot_heads, int n_pivots, int32_t* lists_dev,
                                     int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s);
-cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s);
+cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s,
+                                const int32_t* active = nullptr);
 size_t vslash_scratch_bytes(int n_heads, int N, int chunk);
 cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s);
 cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_rows, const HeadTable& row_of_head,

@@ -253,11 +253,12 @@ __global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float*
 
 // ---- per row: force the diagonal into an empty row, compact the ascending list; one warp per row
 __global__ void compact_rows_kernel(uint8_t* __restrict__ mask, int n_maps, int nb, int32_t* __restrict__ counts,
-                                    int32_t* __restrict__ indices) {
+                                    int32_t* __restrict__ indices, const int32_t* __restrict__ active) {
   const int lane = threadIdx.x & 31;
   const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (w >= (long)n_maps * nb) return;
   const int mp = (int)(w / nb), i = (int)(w % nb);
+  if (active && active[mp] == 0) return;          // a map nobody will read
   uint8_t* row = mask + ((size_t)mp * nb + i) * nb;
   int32_t* irow = indices + ((size_t)mp * nb + i) * nb;
   int cnt = 0;
@@ -388,7 +389,7 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
                                        (int)sizeof(SelShared));
   if (e != cudaSuccess) return e;
   global_select_kernel<<<n_maps, kSelThreads, sizeof(SelShared), s>>>(scores, nb, gamma, mask);
-  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices);
+  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices, nullptr);
   return cudaGetLastError();
 }
 
@@ -465,10 +466,11 @@ cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivo
   return cudaGetLastError();
 }
 
-cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s) {
+cudaError_t launch_compact_rows(uint8_t* mask, int n_maps, int nb, int32_t* counts, int32_t* indices, cudaStream_t s,
+                                const int32_t* active) {
   const long rows = (long)n_maps * nb;
   if (rows == 0) return cudaSuccess;
-  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices);
+  compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices, active);
   return cudaGetLastError();
 }
 

@@ -359,9 +359,10 @@ __global__ void __launch_bounds__(kSelThreads) vector_select_kernel(const float*
 
 // ---- selected lines -> block mask; one CTA per head ----------------------------------------------------
 __global__ void vs_lines_to_mask_kernel(const uint8_t* __restrict__ sel_v, const uint8_t* __restrict__ sel_s, int N, int nb,
-                                        uint8_t* __restrict__ mask) {
+                                        uint8_t* __restrict__ mask, const int32_t* __restrict__ active) {
   __shared__ uint8_t vb[kMaxNb], sb[kMaxNb];
   const int slot = blockIdx.x;
+  if (active && active[slot] == 0) return;
   const uint8_t* sv = sel_v + (size_t)slot * N;
   const uint8_t* ss = sel_s + (size_t)slot * N;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
@@ -433,7 +434,7 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   // a_v and a_s are adjacent: 2 * n_heads vectors of N scores (up() keeps them adjacent when n_heads * N * 4 is a multiple of 256)
   vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a.a_v, v.N, v.gamma, sel, v.active);
   vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
-  vs_lines_to_mask_kernel<<<v.n_heads, 512, 0, s>>>(sel, sel + (size_t)v.n_heads * v.N, v.N, Nb, v.mask);
+  vs_lines_to_mask_kernel<<<v.n_heads, 512, 0, s>>>(sel, sel + (size_t)v.n_heads * v.N, v.N, Nb, v.mask, v.active);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if (v.sel_v_out) {
     if ((e = cudaMemcpyAsync(v.sel_v_out, sel, (size_t)v.n_heads * v.N, cudaMemcpyDeviceToDevice, s)) != cudaSuccess) return e;
@@ -441,7 +442,7 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   if (v.sel_s_out) {
     if ((e = cudaMemcpyAsync(v.sel_s_out, sel + (size_t)v.n_heads * v.N, (size_t)v.n_heads * v.N, cudaMemcpyDeviceToDevice, s)) != cudaSuccess) return e;
   }
-  return launch_compact_rows(v.mask, v.n_heads, Nb, v.counts, v.indices, s);
+  return launch_compact_rows(v.mask, v.n_heads, Nb, v.counts, v.indices, s, v.active);
 }
 
 }  // namespace sp
