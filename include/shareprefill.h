@@ -328,6 +328,48 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
                          float gamma, float delta, float tau, int block, int pooled_construction,
                          sp_tensor* out, uint8_t* mask_out, int32_t* pattern_out, void* stream);
 
+/*
+ * Cross-layer dictionary of pivotal patterns and the layer call that uses it
+ * (Section 5.2: clusters span layers; the first head of a cluster that is met
+ * constructs the pivotal pattern, every later head of the cluster, in this or a
+ * later layer, reuses it after the similarity check).
+ *
+ *   sp_dict_create   a dictionary for up to `max_clusters` cluster ids, layers of
+ *                    `n_q_heads` heads, sequences of `seq` tokens, `block` = 128.
+ *                    It owns device memory for a mask, lists and a representative
+ *                    per cluster plus scratch lists for one layer.
+ *   sp_dict_clear    forget every stored pattern (a new prompt).
+ *   sp_dict_count    clusters that currently have a stored pattern.
+ *
+ *   sp_prefill_attn_layer - one layer of Algorithm "Sparse Attention", heads taken in
+ *   order:
+ *     - a head of the noise cluster (id < 0), or with d_sparse >= delta (highly
+ *       sparse), searches its own vertical-slash pattern;
+ *     - otherwise, if its cluster has a pattern (stored, or constructed by an
+ *       earlier head of this layer), it shares it when d_sim < tau and falls back
+ *       to vertical-slash when not;
+ *     - otherwise it becomes its cluster's pivot: dense attention, pattern
+ *       constructed and stored with its representative (pooled_construction as
+ *       for sp_prefill_attn_auto).
+ *   Who becomes a pivot depends on d_sparse, which is computed on the device: the
+ *   call synchronises `stream` ONCE (a few hundred bytes) before it enqueues the
+ *   rest; the share / vertical-slash decisions stay on the device.
+ *     cluster_of_head  host [n_q_heads]: cluster id in [0, max_clusters) or < 0.
+ *     pattern_out      device i32 [n_q_heads] or NULL: 0 dense (new pivot), 1 shared,
+ *                      2 vertical-slash.  mask_out as for sp_prefill_attn_auto.
+ *   head_dim 128, block 128.  One dictionary serves one context and one sequence
+ *   length; layers must be issued in order on one stream.
+ */
+typedef struct sp_pattern_dict sp_pattern_dict;
+int sp_dict_create(sp_ctx* ctx, int max_clusters, int n_q_heads, int64_t seq, int block, sp_pattern_dict** out);
+int sp_dict_destroy(sp_pattern_dict* dict);
+int sp_dict_clear(sp_pattern_dict* dict);
+int sp_dict_count(const sp_pattern_dict* dict);
+int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q, const sp_tensor* k,
+                          const sp_tensor* v, const int32_t* cluster_of_head, float gamma, float delta,
+                          float tau, int block, int pooled_construction, sp_tensor* out,
+                          uint8_t* mask_out, int32_t* pattern_out, void* stream);
+
 /* Which attention kernel the context launches: 0 = tensor-core kernels
  * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V

@@ -31,6 +31,7 @@ EXPORTS = (
     "sp_prefill_attn", "sp_ctx_set_kernel", "sp_ctx_launch_count", "sp_dense_pivot_attn_fixed_scratch",
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
     "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
+    "sp_dict_create", "sp_dict_destroy", "sp_dict_clear", "sp_dict_count", "sp_prefill_attn_layer",
 )
 
 
@@ -78,6 +79,11 @@ def load() -> ctypes.CDLL:
     lib.sp_determine_pattern.argtypes = [P, T, T, IP, I, I, P, IP, F, F, P, P, P]
     lib.sp_vertical_slash_pattern.argtypes = [P, T, T, IP, I, F, I, P, P, P, P, P, P]
     lib.sp_prefill_attn_auto.argtypes = [P, T, T, T, IP, IP, I, F, F, F, I, I, T, P, P, P]
+    lib.sp_dict_create.argtypes = [P, I, I, ctypes.c_int64, I, ctypes.POINTER(P)]
+    lib.sp_dict_destroy.argtypes = [P]
+    lib.sp_dict_clear.argtypes = [P]
+    lib.sp_dict_count.argtypes = [P]
+    lib.sp_prefill_attn_layer.argtypes = [P, P, T, T, T, IP, F, F, F, I, I, T, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
@@ -245,6 +251,36 @@ class Context:
         _check(self._lib.sp_prefill_attn(self._h, _view(q), _view(k), _view(v), _i32(cluster_map), _i32(pivot_heads),
                                          len(pivot_heads), gamma, block, _view(out), _ptr(mask_out), _stream(stream)),
                "sp_prefill_attn")
+
+
+class PatternDict:
+    """Cross-layer dictionary of pivotal patterns (cluster id -> mask, lists, representative)."""
+
+    def __init__(self, ctx: "Context", max_clusters: int, n_q_heads: int, seq: int, block: int = 128):
+        self._lib, self._ctx = load(), ctx
+        h = ctypes.c_void_p()
+        _check(self._lib.sp_dict_create(ctx._h, max_clusters, n_q_heads, seq, block, ctypes.byref(h)), "sp_dict_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.sp_dict_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def clear(self):
+        _check(self._lib.sp_dict_clear(self._h), "sp_dict_clear")
+
+    def count(self) -> int:
+        return int(self._lib.sp_dict_count(self._h))
+
+    def prefill_attn_layer(self, q, k, v, cluster_of_head, gamma, delta, tau, block, out, pooled_construction=False,
+                           mask_out=None, pattern_out=None, stream=None):
+        cluster_of_head = list(cluster_of_head)
+        _check(self._lib.sp_prefill_attn_layer(self._ctx._h, self._h, _view(q), _view(k), _view(v), _i32(cluster_of_head),
+                                               gamma, delta, tau, block, int(bool(pooled_construction)), _view(out),
+                                               _ptr(mask_out), _ptr(pattern_out), _stream(stream)), "sp_prefill_attn_layer")
 
 
 def _host_ptr(t, dtype, what):

@@ -26,6 +26,20 @@ struct sp_ctx {
   std::vector<cudaEvent_t> events;
 };
 
+// Cross-layer dictionary of pivotal patterns: cluster id -> (mask, compacted lists, representative a~).
+// List slots 0..C-1 belong to the clusters, slots C..C+H-1 are scratch for the vertical-slash lists of a layer.
+struct sp_pattern_dict {
+  int device = 0;
+  int C = 0, H = 0, Nb = 0, B = 0;
+  int64_t N = 0;
+  void* buf = nullptr;
+  uint8_t* masks = nullptr;
+  int32_t* counts = nullptr;
+  int32_t* indices = nullptr;
+  float* a_tilde = nullptr;
+  std::vector<char> has;
+};
+
 namespace {
 
 using namespace sp;
@@ -860,6 +874,222 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
     if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     ctx->launches += 1;
   }
+  return SP_OK;
+}
+
+int sp_dict_create(sp_ctx* ctx, int max_clusters, int n_q_heads, int64_t seq, int block, sp_pattern_dict** out) {
+  if (!ctx || !out || max_clusters <= 0 || n_q_heads <= 0 || seq <= 0) return SP_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (block != 128 || seq % block != 0 || seq / block > kMaxNb || n_q_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  sp_pattern_dict* d = new (std::nothrow) sp_pattern_dict();
+  if (!d) return SP_ERR_WORKSPACE;
+  d->device = ctx->device; d->C = max_clusters; d->H = n_q_heads; d->N = seq; d->B = block; d->Nb = (int)(seq / block);
+  const size_t L = (size_t)d->C + d->H, nn = (size_t)d->Nb * d->Nb;
+  const size_t b_mask = align_up(L * nn), b_counts = align_up(L * d->Nb * sizeof(int32_t)),
+               b_idx = align_up(L * nn * sizeof(int32_t)), b_at = align_up((size_t)d->C * d->Nb * sizeof(float));
+  if (cudaMalloc(&d->buf, b_mask + b_counts + b_idx + b_at) != cudaSuccess) { cudaGetLastError(); delete d; return SP_ERR_WORKSPACE; }
+  char* p = static_cast<char*>(d->buf);
+  d->masks = reinterpret_cast<uint8_t*>(p); p += b_mask;
+  d->counts = reinterpret_cast<int32_t*>(p); p += b_counts;
+  d->indices = reinterpret_cast<int32_t*>(p); p += b_idx;
+  d->a_tilde = reinterpret_cast<float*>(p);
+  d->has.assign(d->C, 0);
+  *out = d;
+  return SP_OK;
+}
+
+int sp_dict_destroy(sp_pattern_dict* d) {
+  if (!d) return SP_OK;
+  DeviceGuard g(d->device);
+  if (d->buf) cudaFree(d->buf);
+  delete d;
+  return SP_OK;
+}
+
+int sp_dict_clear(sp_pattern_dict* d) {
+  if (!d) return SP_ERR_INVALID_ARG;
+  d->has.assign(d->C, 0);
+  return SP_OK;
+}
+
+int sp_dict_count(const sp_pattern_dict* d) {
+  if (!d) return 0;
+  int n = 0;
+  for (char c : d->has) n += c != 0;
+  return n;
+}
+
+int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
+                          const int32_t* cluster_of_head, float gamma, float delta, float tau, int block,
+                          int pooled_construction, sp_tensor* out, uint8_t* mask_out, int32_t* pattern_out, void* stream) {
+  if (!ctx || !dict || !cluster_of_head) return SP_ERR_INVALID_ARG;
+  if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
+  Problem p;
+  int rc = check_problem(q, k, v, out, block, &p);
+  if (rc) return rc;
+  if (p.d != 128 || p.B != 128) return SP_ERR_UNSUPPORTED;
+  if (dict->device != ctx->device || p.Hq > dict->H || p.Nb != dict->Nb || p.B != dict->B) return SP_ERR_INVALID_ARG;
+  for (int h = 0; h < p.Hq; ++h)
+    if (cluster_of_head[h] >= dict->C) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t nn = (size_t)p.Nb * p.Nb;
+
+  // at most one new pivot per cluster of this layer that has no pattern yet
+  int n_new_max = 0;
+  {
+    std::vector<char> seen(dict->C, 0);
+    for (int h = 0; h < p.Hq; ++h) {
+      const int c = cluster_of_head[h];
+      if (c >= 0 && !dict->has[c] && !seen[c]) { seen[c] = 1; ++n_new_max; }
+    }
+  }
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  const size_t o_ahat = take((size_t)p.Hq * p.Nb * sizeof(float));
+  const size_t o_rows = take((size_t)p.Hq * p.Nb * sizeof(float));
+  const size_t o_small = take((size_t)(4 * kMaxHeads) * sizeof(int32_t) + (size_t)kMaxHeads * sizeof(float));
+  const size_t o_imp = take(n_new_max * nn * sizeof(float));
+  const size_t o_scores = take(pooled_construction ? nn * sizeof(float) : 0);
+  const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_new_max, p.Nb, p.d) * sizeof(float)
+                                                    : (size_t)n_new_max * tile_stats_bytes_per_head(p.Nb, p.B));
+  const size_t o_vs = take(vslash_scratch_bytes(p.Hq, p.N, 8));
+  if ((rc = reserve(ctx, off))) return rc;
+  char* ws = static_cast<char*>(ctx->ws);
+  float* a_hat = reinterpret_cast<float*>(ws + o_ahat);
+  float* rows_scratch = reinterpret_cast<float*>(ws + o_rows);
+  int32_t* decide = reinterpret_cast<int32_t*>(ws + o_small);
+  int32_t* lists_dev = decide + kMaxHeads;
+  int32_t* active = lists_dev + kMaxHeads;
+  int32_t* src_dev = active + kMaxHeads;
+  float* d_sparse_dev = reinterpret_cast<float*>(src_dev + kMaxHeads);
+  float* imp = reinterpret_cast<float*>(ws + o_imp);
+
+  // A. Algorithm "Determine Sparse Pattern", first half, for every head: a^ and d_sparse.  The one host
+  //    round trip of the layer: who becomes a pivot depends on d_sparse.
+  int all_heads[kMaxHeads];
+  for (int h = 0; h < p.Hq; ++h) all_heads[h] = h;
+  PooledArgs pa = pooled_args(p, q, k, all_heads, p.Hq);
+  pa.pooled = rows_scratch;
+  if (launch_last_row_distribution(pa, a_hat, s) != cudaSuccess) return SP_ERR_CUDA;
+  if (launch_js_uniform(a_hat, p.Hq, p.Nb, d_sparse_dev, s) != cudaSuccess) return SP_ERR_CUDA;
+  ctx->launches += 3;
+  float d_sparse[kMaxHeads];
+  if (cudaMemcpyAsync(d_sparse, d_sparse_dev, (size_t)p.Hq * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return SP_ERR_CUDA;
+
+  // B. host: heads in order.  Noise cluster or highly sparse -> vertical-slash.  Cluster with a pattern (stored, or
+  //    constructed by an earlier head of this layer) -> candidate for sharing.  Otherwise the head becomes the
+  //    cluster's pivot: dense attention + pattern construction (Algorithm "Share Pivotal Pattern": M = ones).
+  HeadTable piv_heads, piv_slots, member_heads, cand_slot;
+  int n_piv = 0, n_mem = 0;
+  std::vector<char> fresh(dict->C, 0);
+  for (int h = 0; h < p.Hq; ++h) {
+    const int c = cluster_of_head[h];
+    const bool sparse = !(d_sparse[h] < delta);
+    if (c >= 0 && !sparse && !dict->has[c] && !fresh[c]) {
+      fresh[c] = 1;
+      piv_heads.v[n_piv] = h;
+      piv_slots.v[n_piv] = c;
+      ++n_piv;
+      continue;
+    }
+    member_heads.v[n_mem] = h;
+    cand_slot.v[n_mem] = (c >= 0 && !sparse) ? c : -1;
+    ++n_mem;
+  }
+  // the new pivots' representatives a~ are their own a^
+  for (int t = 0; t < n_piv; ++t)
+    if (cudaMemcpyAsync(dict->a_tilde + (size_t)piv_slots.v[t] * p.Nb, a_hat + (size_t)piv_heads.v[t] * p.Nb,
+                        (size_t)p.Nb * sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+      return SP_ERR_CUDA;
+
+  // C. second half of the decision on the device, then lists / flags / codes
+  if (launch_js_pair_decide(a_hat, dict->a_tilde, p.Nb, member_heads, cand_slot, n_mem, tau, decide, s) != cudaSuccess)
+    return SP_ERR_CUDA;
+  if (launch_finalize_layer(decide, cand_slot, member_heads, n_mem, piv_heads, piv_slots, n_piv, dict->C, lists_dev, active,
+                            pattern_out, src_dev, s) != cudaSuccess)
+    return SP_ERR_CUDA;
+  ctx->launches += 2;
+
+  // D. the new pivots: dense attention, pattern into their cluster's slot
+  if (n_piv > 0) {
+    AttnArgs a = base_args(ctx, p, q, k, v, out);
+    a.n_heads = n_piv;
+    for (int t = 0; t < n_piv; ++t) { a.heads.v[t] = piv_heads.v[t]; a.lists.v[t] = -1; }
+    if (!pooled_construction) {
+      a.importance = imp;
+      a.tile_stats = reinterpret_cast<float*>(ws + o_scratch);
+    }
+    if ((rc = launch_attn(ctx, a, s))) return rc;
+    if (pooled_construction) {
+      int ph[kMaxHeads];
+      for (int t = 0; t < n_piv; ++t) ph[t] = piv_heads.v[t];
+      PooledArgs pp = pooled_args(p, q, k, ph, n_piv);
+      pp.qbar = reinterpret_cast<float*>(ws + o_scratch);
+      pp.kbar = pp.qbar + (size_t)n_piv * p.Nb * p.d;
+      pp.diag = pp.kbar + (size_t)n_piv * p.Nb * p.d;
+      pp.pooled = imp;
+      if (launch_pooled_logits(pp, s) != cudaSuccess) return SP_ERR_CUDA;
+      ctx->launches += 2;
+    }
+    for (int t = 0; t < n_piv; ++t) {
+      const int c = piv_slots.v[t];
+      if (pooled_construction) {
+        if (launch_pattern_from_pooled(imp + (size_t)t * nn, 1, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores),
+                                       dict->masks + (size_t)c * nn, dict->counts + (size_t)c * p.Nb,
+                                       dict->indices + (size_t)c * nn, nullptr, s) != cudaSuccess)
+          return SP_ERR_CUDA;
+        ctx->launches += 3;
+      } else {
+        MaskArgs m{imp + (size_t)t * nn, 1, p.Nb, (double)gamma, dict->masks + (size_t)c * nn,
+                   dict->counts + (size_t)c * p.Nb, dict->indices + (size_t)c * nn};
+        if (launch_block_mask(m, s) != cudaSuccess) return SP_ERR_CUDA;
+        ctx->launches += 1;
+      }
+    }
+  }
+
+  // E. vertical-slash search for the heads flagged on the device, block-sparse attention of all members
+  if (n_mem > 0) {
+    VslashArgs vs;
+    memset(&vs, 0, sizeof(vs));
+    vs.chunk = 8;
+    vs.q = static_cast<const __nv_bfloat16*>(q->data);
+    vs.k = static_cast<const __nv_bfloat16*>(k->data);
+    vs.q_sh = q->stride[1]; vs.q_sn = q->stride[2];
+    vs.k_sh = k->stride[1]; vs.k_sn = k->stride[2];
+    vs.n_q_heads = p.Hq; vs.n_kv_heads = p.Hkv; vs.N = p.N; vs.d = p.d; vs.B = p.B; vs.n_heads = n_mem;
+    vs.heads = member_heads;
+    vs.gamma = (double)gamma;
+    vs.scratch = ws + o_vs;
+    vs.mask = dict->masks + (size_t)dict->C * nn;
+    vs.counts = dict->counts + (size_t)dict->C * p.Nb;
+    vs.indices = dict->indices + (size_t)dict->C * nn;
+    vs.active = active;
+    vs.status = ctx->status;
+    if (launch_vertical_slash(vs, s) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 8;
+    AttnArgs b = base_args(ctx, p, q, k, v, out);
+    b.counts = dict->counts;
+    b.indices = dict->indices;
+    b.n_heads = n_mem;
+    for (int t = 0; t < n_mem; ++t) { b.heads.v[t] = member_heads.v[t]; b.lists.v[t] = -1; }
+    b.lists_dev = lists_dev;
+    if ((rc = launch_attn(ctx, b, s))) return rc;
+  }
+  if (mask_out) {
+    HeadTable unused;
+    memset(&unused, 0, sizeof(unused));
+    gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, s>>>(dict->masks, unused, p.Nb, mask_out, src_dev);
+    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
+  }
+  for (int t = 0; t < n_piv; ++t) dict->has[piv_slots.v[t]] = 1;
   return SP_OK;
 }
 

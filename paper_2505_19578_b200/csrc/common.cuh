@@ -98,6 +98,12 @@ cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s);
 cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
                                        uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
                                        cudaStream_t s);
+cudaError_t launch_js_uniform(const float* dist, int n, int nb, float* d_sparse, cudaStream_t s);
+cudaError_t launch_js_pair_decide(const float* a_hat, const float* a_tilde, int nb, const HeadTable& heads,
+                                  const HeadTable& slot_of, int n, float tau, int32_t* decide, cudaStream_t s);
+cudaError_t launch_finalize_layer(const int32_t* decide, const HeadTable& cand_slot, const HeadTable& head_of_member, int n_members,
+                                  const HeadTable& pivot_heads, const HeadTable& pivot_slots, int n_pivots, int vs_base,
+                                  int32_t* lists_dev, int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s);
 cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivot_slot_of_member, const HeadTable& head_of_member,
                                     int n_members, const HeadTable& pivot_heads, int n_pivots, int32_t* lists_dev,
                                     int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s);

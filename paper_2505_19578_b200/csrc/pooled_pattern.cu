@@ -456,6 +456,99 @@ __global__ void finalize_pattern_kernel(const int32_t* __restrict__ decide, Head
 }
 }  // namespace
 
+namespace {
+// sqrt(JSD(a^ || uniform)) of each row of dist [n, nb]; one CTA of 256 threads per row
+__global__ void js_uniform_kernel(const float* __restrict__ dist, int nb, float* __restrict__ d_sparse) {
+  __shared__ float red[8];
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* p_ = dist + (size_t)row * nb;
+  const float u = 1.f / (float)nb;
+  float js = 0.f;
+  for (int j = tid; j < nb; j += blockDim.x) {
+    const float p = p_[j], mm = 0.5f * (p + u);
+    js += (p > 0.f ? p * logf(p / mm) : 0.f) + u * logf(u / mm);
+  }
+  js = warp_sum(js);
+  if (lane == 0) red[warp] = js;
+  __syncthreads();
+  if (tid == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    d_sparse[row] = sqrtf(fmaxf(0.5f * t, 0.f));
+  }
+}
+
+// For each listed head: sqrt(JSD(a^_head || a~_slot)) < tau ?  decide = 0 (share) : 1.  Heads with slot < 0 get 1.
+// a_hat [Hq, nb] indexed by head, a_tilde [n_slots, nb]; one CTA of 256 threads per listed head.
+__global__ void js_pair_decide_kernel(const float* __restrict__ a_hat, const float* __restrict__ a_tilde, int nb,
+                                      HeadTable heads, HeadTable slot_of, float tau, int32_t* __restrict__ decide) {
+  __shared__ float red[8];
+  const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sl = slot_of.v[t];
+  if (sl < 0) { if (tid == 0) decide[t] = 1; return; }
+  const float* p_ = a_hat + (size_t)heads.v[t] * nb;
+  const float* q_ = a_tilde + (size_t)sl * nb;
+  float js = 0.f;
+  for (int j = tid; j < nb; j += blockDim.x) {
+    const float p = p_[j], q = q_[j], mm = 0.5f * (p + q);
+    js += (p > 0.f ? p * logf(p / mm) : 0.f) + (q > 0.f ? q * logf(q / mm) : 0.f);
+  }
+  js = warp_sum(js);
+  if (lane == 0) red[warp] = js;
+  __syncthreads();
+  if (tid == 0) {
+    float s = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+    decide[t] = sqrtf(fmaxf(0.5f * s, 0.f)) < tau ? 0 : 1;
+  }
+}
+
+// lists / flags / codes of a layer driven by the cross-layer dictionary.  Member t: cand_slot >= 0 and decide == 0 ->
+// it walks dictionary slot cand_slot (pattern 1); otherwise its own vertical-slash list vs_base + t (pattern 2).
+__global__ void finalize_layer_kernel(const int32_t* __restrict__ decide, HeadTable cand_slot, HeadTable head_of_member,
+                                      int n_members, HeadTable pivot_heads, HeadTable pivot_slots, int n_pivots, int vs_base,
+                                      int32_t* __restrict__ lists_dev, int32_t* __restrict__ active,
+                                      int32_t* __restrict__ pattern_out, int32_t* __restrict__ src_dev) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n_members) {
+    const int cs = cand_slot.v[t], h = head_of_member.v[t];
+    const bool share = cs >= 0 && decide[t] == 0;
+    const int list = share ? cs : vs_base + t;
+    lists_dev[t] = list;
+    active[t] = share ? 0 : 1;
+    src_dev[h] = list;
+    if (pattern_out) pattern_out[h] = share ? 1 : 2;
+  } else if (t < n_members + n_pivots) {
+    const int p = t - n_members, h = pivot_heads.v[p];
+    src_dev[h] = pivot_slots.v[p];
+    if (pattern_out) pattern_out[h] = 0;
+  }
+}
+}  // namespace
+
+cudaError_t launch_js_uniform(const float* dist, int n, int nb, float* d_sparse, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  js_uniform_kernel<<<n, 256, 0, s>>>(dist, nb, d_sparse);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_js_pair_decide(const float* a_hat, const float* a_tilde, int nb, const HeadTable& heads,
+                                  const HeadTable& slot_of, int n, float tau, int32_t* decide, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  js_pair_decide_kernel<<<n, 256, 0, s>>>(a_hat, a_tilde, nb, heads, slot_of, tau, decide);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_finalize_layer(const int32_t* decide, const HeadTable& cand_slot, const HeadTable& head_of_member, int n_members,
+                                  const HeadTable& pivot_heads, const HeadTable& pivot_slots, int n_pivots, int vs_base,
+                                  int32_t* lists_dev, int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s) {
+  const int n = n_members + n_pivots;
+  if (n == 0) return cudaSuccess;
+  finalize_layer_kernel<<<(n + 127) / 128, 128, 0, s>>>(decide, cand_slot, head_of_member, n_members, pivot_heads, pivot_slots,
+                                                        n_pivots, vs_base, lists_dev, active, pattern_out, src_dev);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_finalize_pattern(const int32_t* decide, const HeadTable& pivot_slot_of_member, const HeadTable& head_of_member,
                                     int n_members, const HeadTable& pivot_heads, int n_pivots, int32_t* lists_dev,
                                     int32_t* active, int32_t* pattern_out, int32_t* src_dev, cudaStream_t s) {

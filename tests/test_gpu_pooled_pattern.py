@@ -324,3 +324,119 @@ def test_prefill_attn_auto_is_the_composition_of_its_steps(binding, name, seq, p
         refo = orc.masked_attention(Q, K, V, h, M, B)
         par.assert_out_close(par.f64(out[h]), refo, f"head {h} (pattern {pat_h[h]})")
     assert torch.isfinite(out.float()).all()
+
+
+# ------------------------------------------------------------------ cross-layer dictionary
+
+def _gap_threshold(values, lo_frac, hi_frac):
+    """A threshold in the middle of the widest gap of the sorted values between two quantiles, so that no value is
+    close to it (distances of order 0.1 .. 0.5 carry an error of about 1e-5 on the GPU)."""
+    v = np.sort(np.asarray(values))
+    lo, hi = int(len(v) * lo_frac), max(int(len(v) * hi_frac), int(len(v) * lo_frac) + 2)
+    w = v[lo:hi + 1]
+    gaps = w[1:] - w[:-1]
+    g = int(np.argmax(gaps))
+    assert gaps[g] > 4e-4, "no clear gap to put a threshold in"
+    return float(0.5 * (w[g] + w[g + 1]))
+
+
+@pytest.mark.parametrize("pooled", [False, True])
+def test_layers_with_cross_layer_dictionary(binding, pooled):
+    from oracle import shareprefill_oracle as orc
+    cfg = synth.scaled(synth.CONFIGS["llama8b_32k"], 2048)
+    B, Nb, Hq, G = cfg.block, cfg.seq // cfg.block, cfg.n_q_heads, cfg.n_q_heads // cfg.n_kv_heads
+    gamma = 0.9
+    layers = [synth.make_layer(cfg, seed=s) for s in (10, 11, 12)]
+    # the second layer attends like the first (same queries and keys, other values), so that its heads find the
+    # first layer's patterns similar; the third is unrelated
+    layers[1] = dict(layers[1], q=layers[0]["q"], k=layers[0]["k"], cluster_map=layers[0]["cluster_map"])
+    cms = []
+    for li, L in enumerate(layers):
+        cm = list(L["cluster_map"])
+        cm[3 + li] = -1                                        # a noise-cluster head in every layer
+        if li == 2:
+            cm = [c if c < 0 else (c + 4) % 10 for c in cm]    # the last layer also brings two clusters not seen before
+        cms.append(cm)
+    # --- reference flow on the oracle's distances
+    a_hats = [[ppo.last_block_distribution(par.f64(L["q"][h]), par.f64(L["k"][h // G]), B) for h in range(Hq)] for L in layers]
+    u = np.full(Nb, 1.0 / Nb)
+    d_sp = [[ppo.js_distance(a, u) for a in row] for row in a_hats]
+    delta = _gap_threshold([x for row in d_sp for x in row], 0.7, 0.95)
+    ref_dict, ref_pat, d_sims = {}, [], []
+    for li in range(3):
+        pats = []
+        for h in range(Hq):
+            c = cms[li][h]
+            if c < 0 or d_sp[li][h] >= delta:
+                pats.append(("vs", None))
+            elif c in ref_dict:
+                d = ppo.js_distance(a_hats[li][h], ref_dict[c][0])
+                d_sims.append(d)
+                pats.append(("cand", d, c))
+            else:
+                ref_dict[c] = (a_hats[li][h], (li, h))
+                pats.append(("pivot", None, c))
+        ref_pat.append(pats)
+    tau = _gap_threshold(d_sims, 0.25, 0.75)
+
+    ctx = binding.Context()
+    d = binding.PatternDict(ctx, 10, Hq, cfg.seq, B)
+    assert d.count() == 0
+    stored = {}                                                # cluster -> mask the GPU stored for it
+    kinds = set()
+    cross_layer = 0
+    for li, L in enumerate(layers):
+        q, k, v = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+        out = torch.full_like(q, float("nan"))
+        mask = torch.full((Hq, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+        pat = torch.full((Hq,), -1, dtype=torch.int32, device="cuda")
+        d.prefill_attn_layer(q, k, v, cms[li], gamma, delta, tau, B, out, pooled_construction=pooled, mask_out=mask, pattern_out=pat)
+        torch.cuda.synchronize()
+        assert ctx.status() == (0, 0)
+        pat_h, mask_h = pat.cpu().numpy(), mask.cpu().numpy()
+        Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
+        tri = np.tril(np.ones((Nb, Nb), np.uint8))
+        vs_heads = [h for h in range(Hq) if pat_h[h] == 2]
+        vmask = torch.empty(len(vs_heads), Nb, Nb, dtype=torch.uint8, device="cuda")
+        vc = torch.empty(len(vs_heads), Nb, dtype=torch.int32, device="cuda")
+        vi = torch.empty(len(vs_heads), Nb, Nb, dtype=torch.int32, device="cuda")
+        ctx.sp_vertical_slash_pattern(q, k, vs_heads, gamma, B, vmask, vc, vi)
+        torch.cuda.synchronize()
+        vmask_h = vmask.cpu().numpy()
+        for h in range(Hq):
+            r = ref_pat[li][h]
+            if r[0] == "pivot":
+                assert pat_h[h] == 0
+                stored[r[2]] = mask_h[h].copy()
+                # the stored pattern is what the construction call gives for this head
+                if pooled:
+                    res = ppo.construct_pivotal_pattern(ppo.pooled_logits(Q[h], K[h // G], B), par.gamma32(gamma))
+                    assert (mask_h[h] != res["mask"]).sum() <= 4
+                else:
+                    I, _ = orc.importance_map(Q, K, V, h, B)
+                    M, _, _, _ = orc.block_mask_from_importance(I, par.gamma32(gamma))
+                    assert (mask_h[h] != M).sum() <= 2
+            elif r[0] == "vs":
+                assert pat_h[h] == 2
+            else:
+                want = 1 if r[1] < tau else 2
+                assert pat_h[h] == want, (li, h, r[1], tau)
+                if want == 1:
+                    assert np.array_equal(mask_h[h], stored[r[2]])       # the pattern of the cluster's pivot, possibly from an earlier layer
+                    cross_layer += int(ref_dict[r[2]][1][0] < li)
+            if pat_h[h] == 2:
+                assert np.array_equal(mask_h[h], vmask_h[vs_heads.index(h)])
+            kinds.add((li, int(pat_h[h])))
+        # outputs under the reported masks
+        picks = {}
+        for h in range(Hq):
+            picks.setdefault(int(pat_h[h]), h)
+        for code, h in picks.items():
+            M = tri if code == 0 else mask_h[h]
+            par.assert_out_close(par.f64(out[h]), orc.masked_attention(Q, K, V, h, M, B), f"layer {li} head {h} pattern {code}")
+        assert torch.isfinite(out.float()).all()
+    assert d.count() == len(ref_dict)
+    assert {0, 1, 2} <= {k_[1] for k_ in kinds}                          # pivots, sharing and vertical-slash all occur
+    assert cross_layer > 0                                               # a pattern stored by one layer is reused by a later one
+    d.clear()
+    assert d.count() == 0
