@@ -294,6 +294,37 @@ def run_ours(args):
         dense_ms = d0.elapsed_time(d1) / 2
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- optional: a stack of layers (each its own seeded inputs and 3-6 clusters), times summed over layers
+    stack = None
+    if rank == 0 and args.stack_layers > 0:
+        import dataclasses
+        import random
+        rng = random.Random(args.seed)
+        t_sparse = t_dense = 0.0
+        piv_counts = []
+        for layer in range(args.stack_layers):
+            lcfg = dataclasses.replace(cfg, n_clusters=rng.randint(3, 6))
+            Ll = synth.make_layer(lcfg, seed=args.seed + 1 + layer, device=str(dev))
+            piv_counts.append(len(Ll["pivot_heads"]))
+            se = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            if layer == 0:                                  # warm the kernels on this shape once
+                ctx.sp_prefill_attn(Ll["q"], Ll["k"], Ll["v"], Ll["cluster_map"], Ll["pivot_heads"], gamma, B, out, stream=stream)
+            torch.cuda.synchronize()
+            se[0].record(stream)
+            ctx.sp_prefill_attn(Ll["q"], Ll["k"], Ll["v"], Ll["cluster_map"], Ll["pivot_heads"], gamma, B, out, stream=stream)
+            se[1].record(stream)
+            if not args.no_dense:
+                ctx.sp_dense_pivot_attn(Ll["q"], Ll["k"], Ll["v"], all_heads, B, out, stream=stream)
+            se[2].record(stream)
+            torch.cuda.synchronize()
+            t_sparse += se[0].elapsed_time(se[1])
+            t_dense += se[1].elapsed_time(se[2])
+            del Ll
+        stack = {"layers": args.stack_layers, "pivots_per_layer": piv_counts, "shareprefill_ms": t_sparse,
+                 "dense_ms": None if args.no_dense else t_dense,
+                 "speedup_vs_dense": None if args.no_dense else t_dense / t_sparse,
+                 "note": "every layer has its own seeded q, k, v and 3-6 clusters (one pivot each); layers treated independently"}
+
     # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
     literal = None
     if rank == 0 and not args.no_literal:
@@ -438,6 +469,7 @@ def run_ours(args):
         "e2e": {"value": layers * F / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "paper_literal_pattern": literal,
+        "layer_stack": stack,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -467,6 +499,8 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--stack-layers", type=int, default=0,
+                    help="also run a stack of this many independent layers (3-6 seeded clusters each) and sum their times")
     ap.add_argument("--no-literal", action="store_true", help="skip the paper-literal pattern construction leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()

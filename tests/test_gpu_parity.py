@@ -196,6 +196,17 @@ def test_prefill_model_shapes_reduced_seq(binding, kernel, name, seq, gamma):
     _check_layer(L, gamma, out, mask)
 
 
+def test_prefill_layer_stack_reduced(binding):
+    # the layer-stack workload: every layer its own seeded inputs and 3..6 clusters (one pivot each), layers independent
+    import dataclasses
+    base = synth.scaled(synth.CONFIGS["llama8b_128k"], 2048)
+    for layer, n_clusters in enumerate((3, 6, 5, 4)):
+        L = synth.make_layer(dataclasses.replace(base, n_clusters=n_clusters), seed=100 + layer)
+        assert len(L["pivot_heads"]) == n_clusters
+        out, mask = _run_layer(binding, L, 0.9, "tc")
+        _check_layer(L, 0.9, out, mask)
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_prefill_degenerate_head_sets(binding, kernel):
     cfg = synth.scaled(synth.CONFIGS["tiny"], 512)
