@@ -13,13 +13,15 @@
 // of Q and of K, so the map needs no pass over the tiles: block means of Q and K
 // (one read of the two tensors), one small product per block, and the diagonal
 // block (only its visible half is averaged) through a running key prefix sum.
-// The global cut is a radix select on the score bits with exact fixed-point bin sums
-// (three passes of 11 + 11 + 10 bits), followed by an ordered pass that breaks
-// ties towards the smaller flattened index.  All of it is HBM- and latency-sized
+// The global cut needs no sort: the cut value is found bit by bit on the score bit
+// patterns with exact fixed-point sums (select.cuh), followed by an ordered pass that
+// breaks ties towards the smaller flattened index.  All of it is HBM- and latency-sized
 // work (a few MB per head).
+#include <cooperative_groups.h>
 #include <math_constants.h>
 
 #include "common.cuh"
+#include "select.cuh"
 
 namespace sp {
 namespace {
@@ -107,148 +109,87 @@ __global__ void pooled_softmax_kernel(const float* __restrict__ pooled, int n_ma
   }
 }
 
-// ---- global cumulative cut over one map; one CTA of 1024 threads per map ---------------------
+// ---- global cumulative cut over one map; a cluster of 8 CTAs of 1024 threads per map --------
+// Rows are dealt round-robin to the cluster's 256 warps (balanced: long and short rows alternate), lanes
+// run along a row's existing blocks j <= i.  Each pass of the cut is a block sum widened to the cluster
+// through distributed shared memory (every CTA reads the eight partial sums and adds them in the same
+// order, so all of them take the same decisions).
 constexpr int kSelThreads = 1024;
-constexpr int kBins = 2048;
+constexpr int kSelCluster = 8;
 
-// Bin sums are kept in 2^-60 fixed point: integer additions commute, so the cut does not depend on
-// the order in which the threads arrive (normalised scores sum to 1: no overflow in 64 bits).
-constexpr double kFix = 1152921504606846976.0;   // 2^60
-
-struct SelShared {
-  unsigned int count[kBins];
-  unsigned long long sum[kBins];
-  double total;
-  unsigned long long cum_above;
-  unsigned int prefix, k_eq, running, select_all;
-  unsigned int warp_cnt[kSelThreads / 32];
-};
-
-__global__ void __launch_bounds__(kSelThreads) global_select_kernel(const float* __restrict__ scores, int nb, double gamma,
-                                                                    uint8_t* __restrict__ mask) {
-  extern __shared__ unsigned char sel_raw[];
-  SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
-  const int mp = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  constexpr int kWarps = kSelThreads / 32;
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+global_select_kernel(const float* __restrict__ scores, int nb, double gamma, uint8_t* __restrict__ mask) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ unsigned long long sh_sum[kSelThreads / 32 + 1];
+  __shared__ unsigned long long partial[2];          // this CTA's sum of the current pass (double-buffered)
+  __shared__ unsigned int row_eq[kMaxNb];            // copies of the cut value per row (every CTA holds all rows)
+  __shared__ unsigned int scan_tmp[kSelThreads / 32];
+  const int mp = blockIdx.y, rank = (int)cluster.block_rank();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kWarps = kSelThreads / 32, kStride = kWarps * kSelCluster;
   const float* sc = scores + (size_t)mp * nb * nb;
   uint8_t* mk = mask + (size_t)mp * nb * nb;
+  const int row0 = rank * kWarps + warp;
 
-  // Rows are dealt to the warps round-robin (balanced: long and short rows alternate), lanes run
-  // along a row's existing blocks j <= i.
+  auto for_each = [&](auto f) {
+    for (int i = row0; i < nb; i += kStride)
+      for (int j = lane; j <= i; j += 32) f(sc[(size_t)i * nb + j]);
+  };
+  int pass = 0;
+  auto widen = [&](unsigned long long x) {
+    const int buf = pass & 1;
+    ++pass;
+    if (tid == 0) partial[buf] = x;
+    cluster.sync();
+    unsigned long long t = 0;
+    for (int r = 0; r < kSelCluster; ++r) t += *cluster.map_shared_rank(&partial[buf], r);
+    return t;
+  };
+  const CutResult cut = block_cumulative_cut<kSelThreads>(for_each, widen, gamma, sh_sum);
 
-  // total of the map (each row sums to 1 up to rounding), float64
-  if (tid == 0) { sh.total = 0.0; sh.cum_above = 0ull; sh.prefix = 0u; sh.select_all = 0u; sh.running = 0u; sh.k_eq = 0u; }
-  __syncthreads();
-  {
-    double t = 0.0;
-    for (int i = warp; i < nb; i += kWarps)
-      for (int j = lane; j <= i; j += 32) t += (double)sc[(size_t)i * nb + j];
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    if (lane == 0) atomicAdd(&sh.total, t);
-  }
-  __syncthreads();
-  const double inv_total = kFix / sh.total;
-  const unsigned long long gamma_fx = gamma >= 4.0 ? ~0ull : __double2ull_rn(gamma * kFix);
-
-  // radix select, most significant digit first: digits of 11, 11, 10 bits
-  const int shift[3] = {21, 10, 0};
-  const int width[3] = {11, 11, 10};
-  for (int pass = 0; pass < 3 && !sh.select_all; ++pass) {
-    for (int b = tid; b < kBins; b += kSelThreads) { sh.count[b] = 0u; sh.sum[b] = 0ull; }
-    __syncthreads();
-    const unsigned int prefix = sh.prefix;
-    const int above = shift[pass] + width[pass];          // bits above this digit
-    const unsigned int dmask = (1u << width[pass]) - 1u;
-    for (int i = warp; i < nb; i += kWarps) {
-      for (int j = lane; j <= i; j += 32) {
-        const float v = sc[(size_t)i * nb + j];
-        const unsigned int bits = __float_as_uint(v);
-        if (pass > 0 && (bits >> above) != prefix) continue;
-        const unsigned int dgt = (bits >> shift[pass]) & dmask;
-        atomicAdd(&sh.count[dgt], 1u);
-        atomicAdd(&sh.sum[dgt], __double2ull_rn((double)v * inv_total));
-      }
-    }
-    __syncthreads();
-    if (tid == 0) {
-      unsigned long long cum = sh.cum_above;
-      int b = (int)dmask;
-      bool found = false;
-      int lowest = -1;                    // lowest non-empty digit seen
-      unsigned long long cum_before_lowest = cum;
-      for (; b >= 0; --b) {
-        if (sh.count[b] == 0u) continue;
-        lowest = b;
-        cum_before_lowest = cum;
-        if (cum + sh.sum[b] >= gamma_fx) { found = true; break; }
-        cum += sh.sum[b];
-      }
-      if (!found && pass > 0 && lowest >= 0) {
-        // cannot happen with exact integer sums; kept as a guard: the cut is the group's smallest value
-        found = true;
-        b = lowest;
-        cum = cum_before_lowest;
-      }
-      if (!found) {
-        sh.select_all = 1u;                       // the scores never reach gamma: every block that exists
-      } else {
-        sh.cum_above = cum;
-        sh.prefix = (prefix << width[pass]) | (unsigned int)b;
-        if (pass == 2) {
-          // prefix is now the bit pattern of the cut value; how many of its copies are needed
-          const unsigned long long v = __double2ull_rn((double)__uint_as_float(sh.prefix) * inv_total);
-          unsigned int k = 0;
-          unsigned long long c = cum;
-          const unsigned int n_eq = sh.count[b];
-          do { c += v; ++k; } while (c < gamma_fx && k < n_eq);
-          sh.k_eq = k;
-        }
-      }
-    }
-    __syncthreads();
-  }
-
-  // marking: everything above the cut value, and the first k_eq copies of it in row-major order.
-  // Groups of kWarps consecutive rows, one row per warp: count the copies per row, prefix over the
-  // group's rows, then mark.
-  const bool all = sh.select_all != 0u;
-  const unsigned int cut = sh.prefix, k_eq = sh.k_eq;
-  for (int i0 = 0; i0 < nb; i0 += kWarps) {
-    const int i = i0 + warp;
-    unsigned int n_eq_row = 0;
-    if (i < nb && !all)
+  // copies of the cut value per row, published to every CTA of the cluster
+  for (int i = tid; i < nb; i += kSelThreads) row_eq[i] = 0u;
+  cluster.sync();
+  if (!cut.all)
+    for (int i = row0; i < nb; i += kStride) {
+      unsigned int n_eq = 0;
       for (int j0 = 0; j0 <= i; j0 += 32) {
         const int j = j0 + lane;
-        const bool eq = j <= i && __float_as_uint(sc[(size_t)i * nb + j]) == cut;
-        n_eq_row += __popc(__ballot_sync(0xffffffffu, eq));
+        n_eq += __popc(__ballot_sync(0xffffffffu, j <= i && score_bits(sc[(size_t)i * nb + j]) == cut.cut_bits));
       }
-    if (lane == 0) sh.warp_cnt[warp] = n_eq_row;
-    __syncthreads();
-    unsigned int rank0 = sh.running;
-    for (int w = 0; w < warp; ++w) rank0 += sh.warp_cnt[w];
-    if (i < nb) {
-      for (int j0 = 0; j0 < nb; j0 += 32) {
-        const int j = j0 + lane;
-        bool on = false;
-        unsigned int bal = 0u;
-        const bool causal = j <= i;
-        unsigned int bits = 0u;
-        if (causal) bits = __float_as_uint(sc[(size_t)i * nb + j]);
-        const bool eq = causal && !all && bits == cut;
-        bal = __ballot_sync(0xffffffffu, eq);
-        if (causal) on = all || bits > cut || (eq && rank0 + __popc(bal & ((1u << lane) - 1u)) < k_eq);
-        if (j < nb) mk[(size_t)i * nb + j] = (uint8_t)(on ? 1 : 0);
-        rank0 += __popc(bal);
-      }
+      if (lane < kSelCluster) *cluster.map_shared_rank(&row_eq[i], lane) = n_eq;
     }
-    __syncthreads();
-    if (tid == 0) {
-      unsigned int t = 0;
-      for (int w = 0; w < kWarps; ++w) t += sh.warp_cnt[w];
-      sh.running += t;
-    }
-    __syncthreads();
+  cluster.sync();
+  // exclusive prefix over the rows (one row per thread, nb <= 1024): rank of a row's first copy in row-major order
+  unsigned int mine = tid < nb ? row_eq[tid] : 0u, incl = mine;
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
   }
+  if (lane == 31) scan_tmp[warp] = incl;
+  __syncthreads();
+  unsigned int base = 0;
+  for (int w = 0; w < warp; ++w) base += scan_tmp[w];
+  __syncthreads();
+  if (tid < nb) row_eq[tid] = base + incl - mine;
+  __syncthreads();
+
+  // marking: everything above the cut value, and the first k_eq copies of it in row-major order
+  for (int i = row0; i < nb; i += kStride) {
+    unsigned int rank0 = row_eq[i];
+    for (int j0 = 0; j0 < nb; j0 += 32) {
+      const int j = j0 + lane;
+      const bool causal = j <= i;
+      const unsigned int bits = causal ? score_bits(sc[(size_t)i * nb + j]) : 0u;
+      const bool eq = causal && !cut.all && bits == cut.cut_bits;
+      const unsigned int bal = __ballot_sync(0xffffffffu, eq);
+      const bool on = causal && (cut.all || bits > cut.cut_bits || (eq && rank0 + __popc(bal & ((1u << lane) - 1u)) < cut.k_eq));
+      if (j < nb) mk[(size_t)i * nb + j] = (uint8_t)(on ? 1 : 0);
+      rank0 += __popc(bal);
+    }
+  }
+  cluster.sync();      // nobody leaves while a neighbour may still read its shared memory
 }
 
 // ---- per row: force the diagonal into an empty row, compact the ascending list; one warp per row
@@ -385,10 +326,7 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
   if (n_maps == 0) return cudaSuccess;
   const long rows = (long)n_maps * nb;
   pooled_softmax_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(pooled, n_maps, nb, scores, last_row);
-  cudaError_t e = cudaFuncSetAttribute(global_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)sizeof(SelShared));
-  if (e != cudaSuccess) return e;
-  global_select_kernel<<<n_maps, kSelThreads, sizeof(SelShared), s>>>(scores, nb, gamma, mask);
+  global_select_kernel<<<dim3(kSelCluster, n_maps), kSelThreads, 0, s>>>(scores, nb, gamma, mask);
   compact_rows_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, s>>>(mask, n_maps, nb, counts, indices, nullptr);
   return cudaGetLastError();
 }

@@ -18,7 +18,7 @@
 //            in shared memory in 2^-40 fixed point (integer adds commute: the
 //            result does not depend on the order of arrival), flushed to global
 //            64-bit counters (each offset receives at most two tiles).
-// Then two cumulative cuts over vectors of N scores (radix select with exact
+// Then two cumulative cuts over vectors of N scores (select.cuh: exact
 // fixed-point sums, ties to the smaller index), and the lines are turned into a
 // block mask: block (i, j), j <= i, is computed if key-block j holds a selected
 // column or a selected offset lies in [(i-j)B - (B-1), (i-j)B + (B-1)].
@@ -27,6 +27,7 @@
 #include <math.h>
 #include <string.h>
 
+#include "select.cuh"
 #include "tc_ptx.cuh"
 
 namespace sp {
@@ -255,103 +256,41 @@ __global__ void vs_slash_to_float_kernel(const unsigned long long* __restrict__ 
 }
 
 // ---- cumulative cut over a vector: minimum descending prefix whose normalised scores reach gamma --------
-constexpr int kSelThreads = 1024, kBins = 2048;
-constexpr double kFix = 1152921504606846976.0;   // 2^60
-
-struct VSel {
-  unsigned int count[kBins];
-  unsigned long long sum[kBins];
-  double total;
-  unsigned long long cum_above;
-  unsigned int prefix, k_eq, running, select_all;
-  unsigned int warp_cnt[kSelThreads / 32];
-};
+constexpr int kSelThreads = 1024;
 
 // grid = n_vectors; vector v at scores + v * n
 __global__ void __launch_bounds__(kSelThreads) vector_select_kernel(const float* __restrict__ scores, long n, double gamma,
                                                                     uint8_t* __restrict__ sel, const int32_t* __restrict__ active) {
   if (active && active[blockIdx.x] == 0) return;
-  extern __shared__ unsigned char vsel_raw[];
-  VSel& sh = *reinterpret_cast<VSel*>(vsel_raw);
+  __shared__ unsigned long long sh_sum[kSelThreads / 32 + 1];
+  __shared__ unsigned int warp_cnt[kSelThreads / 32];
+  __shared__ unsigned int running;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* sc = scores + (size_t)blockIdx.x * n;
   uint8_t* out = sel + (size_t)blockIdx.x * n;
-  auto bits_of = [](float v) { return (v > 0.f && v <= 3.4028235e38f) ? __float_as_uint(v) : 0u; };
-  if (tid == 0) { sh.total = 0.0; sh.cum_above = 0ull; sh.prefix = 0u; sh.select_all = 0u; sh.running = 0u; sh.k_eq = 0u; }
-  __syncthreads();
-  {
-    double t = 0.0;
-    for (long e = tid; e < n; e += kSelThreads) t += (double)__uint_as_float(bits_of(sc[e]));
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    if (lane == 0) atomicAdd(&sh.total, t);
-  }
-  __syncthreads();
-  const double inv_total = sh.total > 0.0 ? kFix / sh.total : 0.0;
-  const unsigned long long gamma_fx = gamma >= 4.0 ? ~0ull : __double2ull_rn(gamma * kFix);
-  const int shift[3] = {21, 10, 0}, width[3] = {11, 11, 10};
-  for (int pass = 0; pass < 3 && !sh.select_all; ++pass) {
-    for (int b = tid; b < kBins; b += kSelThreads) { sh.count[b] = 0u; sh.sum[b] = 0ull; }
-    __syncthreads();
-    const unsigned int prefix = sh.prefix;
-    const int above = shift[pass] + width[pass];
-    const unsigned int dmask = (1u << width[pass]) - 1u;
-    for (long e = tid; e < n; e += kSelThreads) {
-      const unsigned int bits = bits_of(sc[e]);
-      if (pass > 0 && (bits >> above) != prefix) continue;
-      const unsigned int dgt = (bits >> shift[pass]) & dmask;
-      atomicAdd(&sh.count[dgt], 1u);
-      atomicAdd(&sh.sum[dgt], __double2ull_rn((double)__uint_as_float(bits) * inv_total));
-    }
-    __syncthreads();
-    if (tid == 0) {
-      unsigned long long cum = sh.cum_above;
-      int b = (int)dmask, lowest = -1;
-      unsigned long long cum_before_lowest = cum;
-      bool found = false;
-      for (; b >= 0; --b) {
-        if (sh.count[b] == 0u) continue;
-        lowest = b;
-        cum_before_lowest = cum;
-        if (cum + sh.sum[b] >= gamma_fx) { found = true; break; }
-        cum += sh.sum[b];
-      }
-      if (!found && pass > 0 && lowest >= 0) { found = true; b = lowest; cum = cum_before_lowest; }   // guard only
-      if (!found) {
-        sh.select_all = 1u;
-      } else {
-        sh.cum_above = cum;
-        sh.prefix = (prefix << width[pass]) | (unsigned int)b;
-        if (pass == 2) {
-          const unsigned long long v = __double2ull_rn((double)__uint_as_float(sh.prefix) * inv_total);
-          unsigned int k = 0;
-          unsigned long long c = cum;
-          const unsigned int n_eq = sh.count[b];
-          do { c += v; ++k; } while (c < gamma_fx && k < n_eq);
-          sh.k_eq = k;
-        }
-      }
-    }
-    __syncthreads();
-  }
+  auto for_each = [&](auto f) {
+    for (long e = tid; e < n; e += kSelThreads) f(sc[e]);
+  };
+  const CutResult cut = block_cumulative_cut<kSelThreads>(for_each, [](unsigned long long x) { return x; }, gamma, sh_sum);
   // ordered marking: above the cut value, and its first k_eq copies by index
-  const bool all = sh.select_all != 0u;
-  const unsigned int cut = sh.prefix, k_eq = sh.k_eq;
+  if (tid == 0) running = 0u;
+  __syncthreads();
   for (long base = 0; base < n; base += kSelThreads) {
     const long e = base + tid;
-    const unsigned int bits = e < n ? bits_of(sc[e]) : 0u;
-    const bool eq = e < n && !all && bits == cut;
+    const unsigned int bits = e < n ? score_bits(sc[e]) : 0u;
+    const bool eq = e < n && !cut.all && bits == cut.cut_bits;
     const unsigned int bal = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) sh.warp_cnt[warp] = __popc(bal);
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
     __syncthreads();
-    unsigned int before = sh.running;
-    for (int w = 0; w < warp; ++w) before += sh.warp_cnt[w];
+    unsigned int before = running;
+    for (int w = 0; w < warp; ++w) before += warp_cnt[w];
     const unsigned int rank = before + __popc(bal & ((1u << lane) - 1u));
-    if (e < n) out[e] = (uint8_t)((all || bits > cut || (eq && rank < k_eq)) ? 1 : 0);
+    if (e < n) out[e] = (uint8_t)((cut.all || bits > cut.cut_bits || (eq && rank < cut.k_eq)) ? 1 : 0);
     __syncthreads();
     if (tid == 0) {
       unsigned int t = 0;
-      for (int w = 0; w < kSelThreads / 32; ++w) t += sh.warp_cnt[w];
-      sh.running += t;
+      for (int w = 0; w < kSelThreads / 32; ++w) t += warp_cnt[w];
+      running += t;
     }
     __syncthreads();
   }
@@ -424,7 +363,6 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(vs_sweep_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVsSmem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(vs_sweep_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVsSmem)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(vector_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(VSel))) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(a.a_s_fx, 0, (size_t)v.n_heads * v.N * sizeof(unsigned long long), s)) != cudaSuccess) return e;
   vs_sweep_kernel<0><<<dim3(n_chunks, v.n_heads), kVsThreads, kVsSmem, s>>>(a, tq, tk);
   vs_lse_kernel<<<v.n_heads, 128, 0, s>>>(a.partial, n_chunks, a.lse2);
@@ -432,8 +370,8 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   const long n_all = (long)v.n_heads * v.N;
   vs_slash_to_float_kernel<<<(unsigned)((n_all + 255) / 256), 256, 0, s>>>(a.a_s_fx, n_all, a_s);
   // a_v and a_s are adjacent: 2 * n_heads vectors of N scores (up() keeps them adjacent when n_heads * N * 4 is a multiple of 256)
-  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a.a_v, v.N, v.gamma, sel, v.active);
-  vector_select_kernel<<<v.n_heads, kSelThreads, sizeof(VSel), s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
+  vector_select_kernel<<<v.n_heads, kSelThreads, 0, s>>>(a.a_v, v.N, v.gamma, sel, v.active);
+  vector_select_kernel<<<v.n_heads, kSelThreads, 0, s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
   vs_lines_to_mask_kernel<<<v.n_heads, 512, 0, s>>>(sel, sel + (size_t)v.n_heads * v.N, v.N, Nb, v.mask, v.active);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if (v.sel_v_out) {
