@@ -24,6 +24,7 @@
 // column or a selected offset lies in [(i-j)B - (B-1), (i-j)B + (B-1)].
 //
 // Every wait on an mbarrier is bounded (see tc_ptx.cuh).
+#include <cooperative_groups.h>
 #include <math.h>
 #include <string.h>
 
@@ -191,9 +192,13 @@ vs_sweep_kernel(const VsArgs a, const __grid_constant__ CUtensorMap tm_q, const 
             m = m_new;
           }
         } else {
-          // this thread's key against the 128 queries: p = 2^(s - lse) where the key is visible
+          // this thread's key against the 128 queries: p = 2^(s - lse) where the key is visible.
+          // Slash sums: (query r, key x) lies on window index r - x + 127, which (r + 1, x + 1) shares.  A
+          // partial sum travels up the lanes with the queries (lane l hands it to lane l + 1 when the query
+          // advances), so a diagonal is added inside the warp in a fixed order and only the lane where it
+          // leaves the warp touches shared memory: 1 + 1/32 atomics per query and warp instead of 32.
           const int c_glob = j * BLK + x;
-          float colsum = 0.f;
+          float colsum = 0.f, diag = 0.f;
 #pragma unroll 1
           for (int r0 = 0; r0 < BLK; r0 += 32) {
             uint32_t s[32];
@@ -204,10 +209,14 @@ vs_sweep_kernel(const VsArgs a, const __grid_constant__ CUtensorMap tm_q, const 
               float p = ex2_approx(fmaf(__uint_as_float(s[e]), scale, -lse_smem[r]));
               if (j == last && x > r) p = 0.f;
               colsum += p;
-              // offset o = (N - 128 + r) - c_glob lives at window index r - x + 127
-              atomicAdd(&window[r - x + 127], (unsigned long long)__float2ull_rn(p * (float)kSlashFix));
+              const float from_below = __shfl_up_sync(0xffffffffu, diag, 1);
+              diag = p + (lane == 0 ? 0.f : from_below);
+              if (lane == 31)       // the diagonal r - x + 127 has no further key in this warp
+                atomicAdd(&window[r - x + 127], (unsigned long long)__float2ull_rn(diag * (float)kSlashFix));
             }
           }
+          // the diagonals still inside the warp after the last query: lane l holds the one of (127, x)
+          if (lane != 31) atomicAdd(&window[127 - x + 127], (unsigned long long)__float2ull_rn(diag * (float)kSlashFix));
           a.a_v[(size_t)slot * a.N + c_glob] = colsum;
         }
         tc_fence_before();
@@ -256,36 +265,68 @@ __global__ void vs_slash_to_float_kernel(const unsigned long long* __restrict__ 
 }
 
 // ---- cumulative cut over a vector: minimum descending prefix whose normalised scores reach gamma --------
+// A cluster of 4 CTAs per vector, each owning a contiguous quarter; block sums are widened to the cluster
+// through distributed shared memory (every CTA adds the four partial sums in the same order).
 constexpr int kSelThreads = 1024;
+constexpr int kVecCluster = 4;
 
-// grid = n_vectors; vector v at scores + v * n
-__global__ void __launch_bounds__(kSelThreads) vector_select_kernel(const float* __restrict__ scores, long n, double gamma,
-                                                                    uint8_t* __restrict__ sel, const int32_t* __restrict__ active) {
-  if (active && active[blockIdx.x] == 0) return;
+// grid = (kVecCluster, n_vectors); vector v at scores + v * n
+__global__ void __cluster_dims__(kVecCluster, 1, 1) __launch_bounds__(kSelThreads)
+vector_select_kernel(const float* __restrict__ scores, long n, double gamma, uint8_t* __restrict__ sel,
+                     const int32_t* __restrict__ active) {
+  if (active && active[blockIdx.y] == 0) return;           // the whole cluster returns: nobody waits for anybody
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   __shared__ unsigned long long sh_sum[kSelThreads / 32 + 1];
+  __shared__ unsigned long long partial[2];
+  __shared__ unsigned int eq_total[kVecCluster];            // copies of the cut value in each CTA's quarter
   __shared__ unsigned int warp_cnt[kSelThreads / 32];
   __shared__ unsigned int running;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* sc = scores + (size_t)blockIdx.x * n;
-  uint8_t* out = sel + (size_t)blockIdx.x * n;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, rank = (int)cluster.block_rank();
+  const float* sc = scores + (size_t)blockIdx.y * n;
+  uint8_t* out = sel + (size_t)blockIdx.y * n;
+  const long per = (n + kVecCluster - 1) / kVecCluster;
+  const long lo = rank * per, hi = lo + per < n ? lo + per : n;
   auto for_each = [&](auto f) {
-    for (long e = tid; e < n; e += kSelThreads) f(sc[e]);
+    for (long e = lo + tid; e < hi; e += kSelThreads) f(sc[e]);
   };
-  const CutResult cut = block_cumulative_cut<kSelThreads>(for_each, [](unsigned long long x) { return x; }, gamma, sh_sum);
-  // ordered marking: above the cut value, and its first k_eq copies by index
-  if (tid == 0) running = 0u;
+  int pass = 0;
+  auto widen = [&](unsigned long long x) {
+    const int buf = pass & 1;
+    ++pass;
+    if (tid == 0) partial[buf] = x;
+    cluster.sync();
+    unsigned long long t = 0;
+    for (int r = 0; r < kVecCluster; ++r) t += *cluster.map_shared_rank(&partial[buf], r);
+    return t;
+  };
+  const CutResult cut = block_cumulative_cut<kSelThreads>(for_each, widen, gamma, sh_sum);
+
+  // copies of the cut value in the quarters before this one
+  unsigned int n_eq = 0;
+  if (!cut.all)
+    for (long e = lo + tid; e < hi; e += kSelThreads) n_eq += score_bits(sc[e]) == cut.cut_bits;
+  n_eq = (unsigned int)block_sum_u64<kSelThreads>(n_eq, sh_sum);
+  if (tid < kVecCluster) *cluster.map_shared_rank(&eq_total[rank], tid) = n_eq;
+  cluster.sync();
+  if (tid == 0) {
+    unsigned int t = 0;
+    for (int r = 0; r < rank; ++r) t += eq_total[r];
+    running = t;
+  }
   __syncthreads();
-  for (long base = 0; base < n; base += kSelThreads) {
+  // ordered marking: above the cut value, and its first k_eq copies by index
+  for (long base = lo; base < hi; base += kSelThreads) {
     const long e = base + tid;
-    const unsigned int bits = e < n ? score_bits(sc[e]) : 0u;
-    const bool eq = e < n && !cut.all && bits == cut.cut_bits;
+    const unsigned int bits = e < hi ? score_bits(sc[e]) : 0u;
+    const bool eq = e < hi && !cut.all && bits == cut.cut_bits;
     const unsigned int bal = __ballot_sync(0xffffffffu, eq);
     if (lane == 0) warp_cnt[warp] = __popc(bal);
     __syncthreads();
     unsigned int before = running;
     for (int w = 0; w < warp; ++w) before += warp_cnt[w];
-    const unsigned int rank = before + __popc(bal & ((1u << lane) - 1u));
-    if (e < n) out[e] = (uint8_t)((cut.all || bits > cut.cut_bits || (eq && rank < cut.k_eq)) ? 1 : 0);
+    const unsigned int rk = before + __popc(bal & ((1u << lane) - 1u));
+    if (e < hi) out[e] = (uint8_t)((cut.all || bits > cut.cut_bits || (eq && rk < cut.k_eq)) ? 1 : 0);
     __syncthreads();
     if (tid == 0) {
       unsigned int t = 0;
@@ -294,6 +335,7 @@ __global__ void __launch_bounds__(kSelThreads) vector_select_kernel(const float*
     }
     __syncthreads();
   }
+  cluster.sync();      // nobody leaves while a neighbour may still read its shared memory
 }
 
 // ---- selected lines -> block mask; one CTA per head ----------------------------------------------------
@@ -317,10 +359,8 @@ __global__ void vs_lines_to_mask_kernel(const uint8_t* __restrict__ sel_v, const
   }
   __syncthreads();
   uint8_t* m = mask + (size_t)slot * nb * nb;
-  for (long e = threadIdx.x; e < (long)nb * nb; e += blockDim.x) {
-    const int i = (int)(e / nb), j = (int)(e % nb);
-    m[e] = (uint8_t)((j <= i && (vb[j] || sb[i - j])) ? 1 : 0);
-  }
+  for (int i = warp; i < nb; i += n_warps)
+    for (int j = lane; j < nb; j += 32) m[(size_t)i * nb + j] = (uint8_t)((j <= i && (vb[j] || sb[i - j])) ? 1 : 0);
 }
 
 }  // namespace
@@ -370,8 +410,8 @@ cudaError_t launch_vertical_slash(const VslashArgs& v, cudaStream_t s) {
   const long n_all = (long)v.n_heads * v.N;
   vs_slash_to_float_kernel<<<(unsigned)((n_all + 255) / 256), 256, 0, s>>>(a.a_s_fx, n_all, a_s);
   // a_v and a_s are adjacent: 2 * n_heads vectors of N scores (up() keeps them adjacent when n_heads * N * 4 is a multiple of 256)
-  vector_select_kernel<<<v.n_heads, kSelThreads, 0, s>>>(a.a_v, v.N, v.gamma, sel, v.active);
-  vector_select_kernel<<<v.n_heads, kSelThreads, 0, s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
+  vector_select_kernel<<<dim3(kVecCluster, v.n_heads), kSelThreads, 0, s>>>(a.a_v, v.N, v.gamma, sel, v.active);
+  vector_select_kernel<<<dim3(kVecCluster, v.n_heads), kSelThreads, 0, s>>>(a_s, v.N, v.gamma, sel + (size_t)v.n_heads * v.N, v.active);
   vs_lines_to_mask_kernel<<<v.n_heads, 512, 0, s>>>(sel, sel + (size_t)v.n_heads * v.N, v.N, Nb, v.mask, v.active);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if (v.sel_v_out) {
