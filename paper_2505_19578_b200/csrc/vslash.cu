@@ -16,8 +16,9 @@
 //            one key column: p = exp(s - lse) down the column gives a_v directly
 //            (one writer per key), and the slash sums go through a 255-entry window
 //            in shared memory in 2^-40 fixed point (integer adds commute: the
-//            result does not depend on the order of arrival), flushed to global
-//            64-bit counters (each offset receives at most two tiles).
+//            result does not depend on the order of arrival) that slides along with
+//            the key-blocks of a chunk; finished offsets are stored, and only the
+//            two ends of a chunk are added atomically to global 64-bit counters.
 // Then two cumulative cuts over vectors of N scores (select.cuh: exact
 // fixed-point sums, ties to the smaller index), and the lines are turned into a
 // block mask: block (i, j), j <= i, is computed if key-block j holds a selected
@@ -192,13 +193,9 @@ vs_sweep_kernel(const VsArgs a, const __grid_constant__ CUtensorMap tm_q, const 
             m = m_new;
           }
         } else {
-          // this thread's key against the 128 queries: p = 2^(s - lse) where the key is visible.
-          // Slash sums: (query r, key x) lies on window index r - x + 127, which (r + 1, x + 1) shares.  A
-          // partial sum travels up the lanes with the queries (lane l hands it to lane l + 1 when the query
-          // advances), so a diagonal is added inside the warp in a fixed order and only the lane where it
-          // leaves the warp touches shared memory: 1 + 1/32 atomics per query and warp instead of 32.
+          // this thread's key against the 128 queries: p = 2^(s - lse) where the key is visible
           const int c_glob = j * BLK + x;
-          float colsum = 0.f, diag = 0.f;
+          float colsum = 0.f;
 #pragma unroll 1
           for (int r0 = 0; r0 < BLK; r0 += 32) {
             uint32_t s[32];
@@ -209,29 +206,40 @@ vs_sweep_kernel(const VsArgs a, const __grid_constant__ CUtensorMap tm_q, const 
               float p = ex2_approx(fmaf(__uint_as_float(s[e]), scale, -lse_smem[r]));
               if (j == last && x > r) p = 0.f;
               colsum += p;
-              const float from_below = __shfl_up_sync(0xffffffffu, diag, 1);
-              diag = p + (lane == 0 ? 0.f : from_below);
-              if (lane == 31)       // the diagonal r - x + 127 has no further key in this warp
-                atomicAdd(&window[r - x + 127], (unsigned long long)__float2ull_rn(diag * (float)kSlashFix));
+              // offset o = (N - 128 + r) - c_glob lives at window index r - x + 127
+              atomicAdd(&window[r - x + 127], (unsigned long long)__float2ull_rn(p * (float)kSlashFix));
             }
           }
-          // the diagonals still inside the warp after the last query: lane l holds the one of (127, x)
-          if (lane != 31) atomicAdd(&window[127 - x + 127], (unsigned long long)__float2ull_rn(diag * (float)kSlashFix));
           a.a_v[(size_t)slot * a.N + c_glob] = colsum;
         }
         tc_fence_before();
         mbar_arrive(bar(VB_S_EMPTY + st));
       }
       if (SWEEP == 1) {
-        // flush the window: offsets o_base .. o_base + 254
+        // The window covers offsets o_base .. o_base + 254 and moves down by 128 with every key-block: its
+        // upper 128 entries are final once this tile is in (they also hold the previous tile's share, carried
+        // over below) and are written out; its lower 127 entries are carried to the next tile.  Only the ends of
+        // a chunk meet another CTA's tiles and need atomic adds.
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const long o_base = (long)(a.N - BLK) - (long)j * BLK - 127;
-        for (int idx = x; idx < 255; idx += 128) {
+        unsigned long long* dst = a.a_s_fx + (size_t)slot * a.N;
+        {
+          const int idx = 127 + x;
           const unsigned long long wv = window[idx];
           const long o = o_base + idx;
-          if (wv != 0ull && o >= 0 && o < a.N) atomicAdd(&a.a_s_fx[(size_t)slot * a.N + o], wv);
-          window[idx] = 0ull;
+          if (o >= 0 && o < a.N) {
+            if (t == 0) { if (wv != 0ull) atomicAdd(&dst[o], wv); }
+            else dst[o] = wv;
+          }
         }
+        const unsigned long long carry = x < 127 ? window[x] : 0ull;
+        if (t == n_tiles - 1 && x < 127) {
+          const long o = o_base + x;
+          if (carry != 0ull && o >= 0 && o < a.N) atomicAdd(&dst[o], carry);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        window[x] = 0ull;
+        if (x < 127) window[x + 128] = (t == n_tiles - 1) ? 0ull : carry;
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
     }
