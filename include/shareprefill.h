@@ -214,8 +214,9 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
 
 /*
  * The whole layer with HOST buffers: the same steps as sp_prefill_attn (same
- * algorithms of the paper), with the transfers pipelined around them.  K, V and
- * the pivots' queries are copied in first; the pivots' dense attention and the
+ * algorithms of the paper), with the transfers pipelined around them.  The K and V
+ * of the pivots' KV heads and the pivots' queries are copied in first, then the
+ * other KV heads; the pivots' dense attention and the
  * mask construction run while the members' queries are still arriving; the
  * members run in groups of four heads, each group's outputs copied back while
  * the next group computes.  Copies use two streams owned by the context; when the

@@ -541,13 +541,27 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
   // this context may still be reading the device copies).
   if (!hand_over(sc, sin) || !hand_over(sc, sout)) return SP_ERR_CUDA;
 
-  // in: K, V, the pivots' queries; compute: step 1 + step 2 while the members' queries arrive
-  if (cudaMemcpyAsync(dk, k_host, (size_t)n_kv_heads * head_bytes, cudaMemcpyHostToDevice, sin) != cudaSuccess ||
-      cudaMemcpyAsync(dv, v_host, (size_t)n_kv_heads * head_bytes, cudaMemcpyHostToDevice, sin) != cudaSuccess)
-    return SP_ERR_CUDA;
-  for (int t = 0; t < n_pivots; ++t)
+  // in: first what the pivots need (their KV heads' K and V, their queries) so that step 1 starts as early as
+  // possible; then the other KV heads; the members' queries follow in groups while steps 1 and 2 compute
+  const char* hk = static_cast<const char*>(k_host);
+  const char* hv = static_cast<const char*>(v_host);
+  auto copy_in_kv = [&](int gkv) {
+    return cudaMemcpyAsync(dk + (size_t)gkv * head_bytes, hk + (size_t)gkv * head_bytes, head_bytes, cudaMemcpyHostToDevice, sin) == cudaSuccess &&
+           cudaMemcpyAsync(dv + (size_t)gkv * head_bytes, hv + (size_t)gkv * head_bytes, head_bytes, cudaMemcpyHostToDevice, sin) == cudaSuccess;
+  };
+  bool kv_sent[kMaxHeads];
+  for (int gkv = 0; gkv < n_kv_heads; ++gkv) kv_sent[gkv] = false;
+  const int group = n_q_heads / n_kv_heads;
+  for (int t = 0; t < n_pivots; ++t) {
+    const int gkv = pivot_heads[t] / group;
+    if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return SP_ERR_CUDA; kv_sent[gkv] = true; }
     if (!copy_in_head(pivot_heads[t])) return SP_ERR_CUDA;
-  if (!hand_over(sin, sc)) return SP_ERR_CUDA;
+  }
+  if (!hand_over(sin, sc)) return SP_ERR_CUDA;                      // step 1 may start
+  for (int gkv = 0; gkv < n_kv_heads; ++gkv)
+    if (!kv_sent[gkv] && !copy_in_kv(gkv)) return SP_ERR_CUDA;
+  cudaEvent_t all_kv = event();
+  if (!all_kv || cudaEventRecord(all_kv, sin) != cudaSuccess) return SP_ERR_CUDA;
 
   AttnArgs a = base_args(ctx, p, &q, &k, &v, &o);
   a.n_heads = n_pivots;
@@ -576,6 +590,7 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
     ++n_members;
   }
   constexpr int kGroup = 4;
+  if (cudaStreamWaitEvent(sc, all_kv, 0) != cudaSuccess) return SP_ERR_CUDA;     // members read every KV head
   for (int g0 = 0; g0 < n_members; g0 += kGroup) {
     const int g1 = g0 + kGroup < n_members ? g0 + kGroup : n_members;
     for (int x = g0; x < g1; ++x)
