@@ -440,3 +440,49 @@ def test_layers_with_cross_layer_dictionary(binding, pooled):
     assert cross_layer > 0                                               # a pattern stored by one layer is reused by a later one
     d.clear()
     assert d.count() == 0
+
+
+# ------------------------------------------------------------------ argument checking of these calls (host side)
+
+def test_invalid_arguments_of_the_pattern_calls(binding):
+    ctx = binding.Context()
+    q = torch.zeros(4, 512, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(2, 512, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(q)
+    Nb = 4
+    f = torch.zeros(1, Nb, Nb, device="cuda")
+    m = torch.zeros(1, Nb, Nb, dtype=torch.uint8, device="cuda")
+    c = torch.zeros(1, Nb, dtype=torch.int32, device="cuda")
+    ix = torch.zeros(1, Nb, Nb, dtype=torch.int32, device="cuda")
+    pat = torch.zeros(4, dtype=torch.int32, device="cuda")
+
+    def code(fn):
+        with pytest.raises(binding.SpError) as e:
+            fn()
+        return e.value.code
+
+    INV, UNS = binding.SP_ERR_INVALID_ARG, binding.SP_ERR_UNSUPPORTED
+    assert code(lambda: ctx.sp_pooled_logits(q, k, [4], 128, f)) == INV                    # head range
+    assert code(lambda: ctx.sp_pooled_logits(q, k, [0], 96, f)) == UNS                     # block
+    assert code(lambda: ctx.sp_pattern_from_pooled(f, 0.0, m, c, ix)) == INV               # gamma
+    assert code(lambda: ctx.sp_pattern_from_pooled(f, 0.9, None, c, ix)) == INV            # the mask is required
+    assert code(lambda: ctx.sp_determine_pattern(q, k, [0], 128, None, [0], 0.3, 0.2, pat)) == INV
+    assert code(lambda: ctx.sp_vertical_slash_pattern(q, k, [0], -1.0, 128, m, c, ix)) == INV
+    q64 = torch.zeros(4, 512, 64, dtype=torch.bfloat16, device="cuda")
+    k64 = torch.zeros(2, 512, 64, dtype=torch.bfloat16, device="cuda")
+    o64 = torch.zeros_like(q64)
+    assert code(lambda: ctx.sp_vertical_slash_pattern(q64, k64, [0], 0.9, 64, m, c, ix)) == UNS
+    assert code(lambda: ctx.sp_prefill_attn_auto(q, k, k, [0, 0, 1, 1], [0, 0], 0.9, 0.3, 0.2, 128, out)) == INV
+    assert code(lambda: ctx.sp_prefill_attn_auto(q64, k64, k64, [0, 0, 1, 1], [0], 0.9, 0.3, 0.2, 64, o64)) == UNS
+    d = binding.PatternDict(ctx, 2, 4, 512, 128)
+    assert code(lambda: d.prefill_attn_layer(q, k, k, [0, 1, 2, 0], 0.9, 0.3, 0.2, 128, out)) == INV      # cluster id
+    q2 = torch.zeros(4, 1024, 128, dtype=torch.bfloat16, device="cuda")
+    k2 = torch.zeros(2, 1024, 128, dtype=torch.bfloat16, device="cuda")
+    o2 = torch.zeros_like(q2)
+    assert code(lambda: d.prefill_attn_layer(q2, k2, k2, [0, 1, 0, 1], 0.9, 0.3, 0.2, 128, o2)) == INV    # other length
+    with pytest.raises(binding.SpError):
+        binding.PatternDict(ctx, 2, 4, 500, 128)
+    with pytest.raises(ValueError):                                                        # host call wants host tensors
+        ctx.sp_prefill_attn_host(q, k.cpu(), k.cpu(), [0, 0, 1, 1], [0], 0.9, 128, out.cpu())
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
