@@ -38,6 +38,14 @@ if ROOT not in sys.path:
 
 from paper_2505_19578_b200 import synth  # noqa: E402
 
+# DRAM bytes (read + write) per launch of the attention kernel from an ncu capture of this very workload
+# (profiles/attn_pair_kernel_llama8b_128k_dram_traffic.md); valid for the default workload, gamma and seed only,
+# and to be set back to None whenever the attention kernel changes.
+NCU_DRAM_TRAFFIC = {
+    ("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 1962653952 + 1182885376,
+    ("llama8b_128k", 131072, 0.9, 0, "block_sparse_attn"): 7030535680 + 901785344,
+}
+
 METRIC = "effective_tflops_prefill_attention_layer"
 UNIT = "TFLOP/s"
 
@@ -439,7 +447,9 @@ def run_ours(args):
         "peak": peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], "unit": "TFLOP/s",
         "frac": dom[2] / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
         "peak_kind": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
-        "frac_of_burst_peak": dom[2] / peaks["bf16_tflops"], "traffic": None,
+        "frac_of_burst_peak": dom[2] / peaks["bf16_tflops"],
+        "traffic": NCU_DRAM_TRAFFIC.get((cfg.name, cfg.seq, round(gamma, 6), args.seed, dom[0])),
+        "traffic_unit": "bytes of DRAM read + write per launch (ncu, same workload)",
         "ms_per_launch": dom[1], "flops_per_launch": (pivot_tiles if dom[0].startswith("pivot") else member_tiles) * Ft,
         "timing": "CUDA events around each of the three public calls, same inputs, same number of steps",
     }
