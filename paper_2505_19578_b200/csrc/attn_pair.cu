@@ -174,8 +174,19 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_pairs = (a.Nb + 1) >> 1;
-  const int u = n_pairs - 1 - (int)blockIdx.y;      // long row-blocks first, across all heads
-  const int slot = blockIdx.x;
+  // Work order: the heads of one KV head together (their K/V set, 64 MB at 128K, stays in L2 while they run),
+  // inside such a group the longest row-block pairs first, heads fastest.
+  int slot, u;
+  {
+    int id = (int)blockIdx.x, g = 0;
+    while (g + 1 < a.n_groups && id >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
+      id -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
+      ++g;
+    }
+    const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
+    slot = a.order.v[a.group_start.v[g] + id % ng];
+    u = n_pairs - 1 - id / ng;
+  }
   const int h = a.heads.v[slot];
   const int g = h / a.group;
   const int list = a.lists_dev ? a.lists_dev[slot] : a.lists.v[slot];   // decided on the device, or by the host
@@ -197,7 +208,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   const bool emit = a.importance != nullptr && list < 0;
   const Abort ab{abort_flag, a.status};
   // Optional phase trace (one CTA, one thread per role): {(event << 32) | step, SM clock} pairs.
-  const bool tracing = a.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0;
+  const bool tracing = a.trace != nullptr && blockIdx.x == 0;
   int trace_n = 0;
   auto trace = [&](int role, int event, int step) {
     if (tracing && trace_n < a.trace_cap) {
@@ -592,8 +603,19 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 
 bool attn_pair_supported(const AttnArgs& a) { return a.d == D && a.B == BLK; }
 
-cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s) {
-  if (!attn_pair_supported(a)) return cudaErrorInvalidValue;
+cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
+  if (!attn_pair_supported(a_in)) return cudaErrorInvalidValue;
+  AttnArgs a = a_in;
+  // slots sorted by KV head (stable), and where each KV head's group starts
+  int n = 0;
+  a.n_groups = 0;
+  for (int g = 0; g < a.n_kv_heads; ++g) {
+    const int start = n;
+    for (int t = 0; t < a.n_heads; ++t)
+      if (a.heads.v[t] / a.group == g) a.order.v[n++] = t;
+    if (n > start) a.group_start.v[a.n_groups++] = start;
+  }
+  a.group_start.v[a.n_groups] = n;
   CUtensorMap tq, tk, tv;
   if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
       !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK) ||
@@ -601,7 +623,7 @@ cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s) {
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
   if (e != cudaSuccess) return e;
-  attn_pair_kernel<<<dim3(a.n_heads, (a.Nb + 1) / 2), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
+  attn_pair_kernel<<<a.n_heads * ((a.Nb + 1) / 2), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
   return cudaGetLastError();
 }
 

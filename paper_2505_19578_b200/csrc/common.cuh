@@ -30,6 +30,9 @@ struct AttnArgs {
   HeadTable heads;         // query-head index per slot
   HeadTable lists;         // list index per slot, -1 = dense (all causal tiles)
   const int32_t* lists_dev;  // if not null: list index per slot read from device memory instead
+  HeadTable order;         // paired kernel: slots sorted by KV head (position -> slot)
+  HeadTable group_start;   // paired kernel: first sorted position of each KV-head group, then n_heads
+  int n_groups;
   const int32_t* counts;   // [n_lists, Nb]       (may be null when every slot is dense)
   const int32_t* indices;  // [n_lists, Nb, Nb]
   float* importance;       // [n_heads, Nb, Nb] or null
