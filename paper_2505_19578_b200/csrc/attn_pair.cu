@@ -606,14 +606,27 @@ bool attn_pair_supported(const AttnArgs& a) { return a.d == D && a.B == BLK; }
 cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
   if (!attn_pair_supported(a_in)) return cudaErrorInvalidValue;
   AttnArgs a = a_in;
-  // slots sorted by KV head (stable), and where each KV head's group starts
+  // Work order.  Many CTAs (forty waves or more): the slots sorted by KV head (stable), one group per KV head,
+  // so that a K/V set stays in L2 while its heads run.  Fewer: one group, i.e. the longest pairs of all heads
+  // first, because with a few waves the balance of the last wave matters more than L2.
+  int n_sm = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const bool by_kv_head = (long)a.n_heads * ((a.Nb + 1) / 2) >= 40L * n_sm;
   int n = 0;
   a.n_groups = 0;
-  for (int g = 0; g < a.n_kv_heads; ++g) {
-    const int start = n;
-    for (int t = 0; t < a.n_heads; ++t)
-      if (a.heads.v[t] / a.group == g) a.order.v[n++] = t;
-    if (n > start) a.group_start.v[a.n_groups++] = start;
+  if (by_kv_head) {
+    for (int g = 0; g < a.n_kv_heads; ++g) {
+      const int start = n;
+      for (int t = 0; t < a.n_heads; ++t)
+        if (a.heads.v[t] / a.group == g) a.order.v[n++] = t;
+      if (n > start) a.group_start.v[a.n_groups++] = start;
+    }
+  } else {
+    for (int t = 0; t < a.n_heads; ++t) a.order.v[n++] = t;
+    a.group_start.v[a.n_groups++] = 0;
   }
   a.group_start.v[a.n_groups] = n;
   CUtensorMap tq, tk, tv;
