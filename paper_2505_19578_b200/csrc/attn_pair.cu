@@ -229,7 +229,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(BAR_S_FULL + x), 1);
-      mbar_init(bar(BAR_P_FULL + x), 128);
+      mbar_init(bar(BAR_P_FULL + x), 4);      // one arrival per softmax warp
       mbar_init(bar(BAR_O_DONE + x), 1);
     }
     *abort_flag = 0;
@@ -521,7 +521,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       if (tthread) trace(trole, 13, t);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar(BAR_P_FULL + x));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_P_FULL + x));
       if (tthread) trace(trole, 15, t);
       // off the critical path: running sum and the tile statistic
       l += tile_sum;
