@@ -256,6 +256,35 @@ def test_prefill_host_buffers_equal_device_call(binding, name, seq):
     assert torch.equal(pout.view(torch.int16), out_d.cpu().view(torch.int16))
 
 
+@pytest.mark.parametrize("cm,pivots", [
+    ([0, 0, 0, 1, 1, -1, 2, 0], [2, 0, 3]),      # unclustered head, cluster without pivot, two pivots in one cluster
+    ([0, 0, 0, 0, 0, 0, 0, 0], [5]),             # a single pivot: nothing is held back
+    ([0, 1, 0, 1, 0, 1, 0, 1], []),              # no pivot at all: every head runs dense
+    ([0, 1, 2, 3, 0, 1, 2, 3], [3, 2, 1, 0]),    # the last pivot's cluster goes after the other clusters' members
+    (None, None),                                # head_dim 128 (paired kernel): pivots reversed, one cluster left without
+])
+def test_prefill_host_buffers_irregular_cluster_tables(binding, cm, pivots):
+    # the host-buffer call orders pivots, clusters and copies differently from the device call; same bits out
+    if cm is None:
+        L = synth.make_layer(synth.scaled(synth.CONFIGS["llama8b_32k"], 2048), seed=9)
+        cm, pivots = L["cluster_map"], list(reversed(L["pivot_heads"]))[:-1]
+    else:
+        L = synth.make_layer(synth.scaled(synth.CONFIGS["tiny"], 1024), seed=9)
+    cfg = L["cfg"]
+    Nb = cfg.seq // cfg.block
+    L2 = dict(L, cluster_map=cm, pivot_heads=pivots)
+    out_d, mask_d = _run_layer(binding, L2, 0.9, "tc")
+    _check_layer(L2, 0.9, out_d, mask_d)
+    ctx = binding.Context()
+    hq, hk, hv = (L[x].contiguous().pin_memory() for x in ("q", "k", "v"))
+    hout = torch.full(hq.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    hmask = torch.full((cfg.n_q_heads, Nb, Nb), 9, dtype=torch.uint8).pin_memory()
+    ctx.sp_prefill_attn_host(hq, hk, hv, cm, pivots, 0.9, cfg.block, hout, mask_out=hmask)
+    _sync_ok(ctx)
+    assert torch.equal(hout.view(torch.int16), out_d.cpu().view(torch.int16))
+    assert torch.equal(hmask, mask_d.cpu())
+
+
 def test_tc_and_simt_kernels_agree_on_importance(binding):
     # two different algorithms for the tile mass (one pass + spilled statistics vs two passes)
     q, k, v = _rand_layer(7, 2, 1, 1024, 128, scale=3.0)
