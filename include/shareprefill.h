@@ -90,6 +90,16 @@ int sp_ctx_reserve(sp_ctx* ctx, size_t bytes);
  * the wait that gave up (kernel-internal id).  Either pointer may be NULL. */
 int sp_get_status(sp_ctx* ctx, int* code /* host, out */, int* where /* host, out */);
 
+/* Self-test of the bounded device-side waits: launches one warp that waits,
+ * for at most `limit_cycles` SM cycles (1 .. 2e9), on a barrier nothing arrives
+ * at.  The wait runs out, the kernel returns normally, and after the caller has
+ * synchronised sp_get_status reports SP_ERR_TIMEOUT with where = 99.  Until
+ * sp_get_status has cleared the status word every kernel of this context does
+ * no work (outputs are left untouched), exactly as after a real timeout.  No
+ * device fault, trap or unbounded loop is involved.  The paper has no
+ * counterpart; this exists so that the failure path can be tested. */
+int sp_selftest_wait_timeout(sp_ctx* ctx, int64_t limit_cycles, void* stream);
+
 /* Static string for an SP_* code. */
 const char* sp_strerror(int code);
 

@@ -32,6 +32,7 @@ EXPORTS = (
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
     "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
     "sp_dict_create", "sp_dict_destroy", "sp_dict_clear", "sp_dict_count", "sp_prefill_attn_layer",
+    "sp_selftest_wait_timeout",
 )
 
 
@@ -85,6 +86,7 @@ def load() -> ctypes.CDLL:
     lib.sp_dict_count.argtypes = [P]
     lib.sp_prefill_attn_layer.argtypes = [P, P, T, T, T, IP, F, F, F, I, I, T, P, P, P]
     lib.sp_ctx_set_kernel.argtypes = [P, I]
+    lib.sp_selftest_wait_timeout.argtypes = [P, ctypes.c_int64, P]
     lib.sp_ctx_set_trace.argtypes = [P, P, I]
     lib.sp_ctx_launch_count.argtypes = [P]
     lib.sp_ctx_launch_count.restype = ctypes.c_int64
@@ -158,6 +160,10 @@ class Context:
         """events: zeroed CUDA int64 tensor of 5 * events_per_role * 2 entries, or None to switch off."""
         _check(self._lib.sp_ctx_set_trace(self._h, _ptr(events), events_per_role if events is not None else 0),
                "sp_ctx_set_trace")
+
+    def selftest_wait_timeout(self, limit_cycles: int, stream=None):
+        """Launch the one-warp kernel whose wait cannot complete (see the header); status() then reports the timeout."""
+        _check(self._lib.sp_selftest_wait_timeout(self._h, int(limit_cycles), _stream(stream)), "sp_selftest_wait_timeout")
 
     def launch_count(self) -> int:
         return int(self._lib.sp_ctx_launch_count(self._h))

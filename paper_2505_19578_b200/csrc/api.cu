@@ -257,6 +257,16 @@ int sp_get_status(sp_ctx* ctx, int* code, int* where) {
   return SP_OK;
 }
 
+int sp_selftest_wait_timeout(sp_ctx* ctx, int64_t limit_cycles, void* stream) {
+  if (!ctx || limit_cycles <= 0 || limit_cycles > 2000000000ll) return SP_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SP_ERR_CUDA;
+  if (launch_wait_selftest(ctx->status, (long long)limit_cycles, 99, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SP_ERR_CUDA;
+  ctx->launches += 1;
+  return SP_OK;
+}
+
 int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
   if (!ctx || which < 0 || which > 2) return SP_ERR_INVALID_ARG;
   ctx->kernel = which;

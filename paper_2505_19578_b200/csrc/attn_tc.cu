@@ -396,4 +396,28 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s) {
   return cudaErrorInvalidValue;
 }
 
+namespace {
+// One warp waits, with the given cycle limit, on an mbarrier that nothing ever arrives at: the wait runs out, the
+// status word gets SP_ERR_TIMEOUT and the location id, and the kernel returns normally.
+__global__ void wait_selftest_kernel(int* status, long long limit_cycles, int where) {
+  __shared__ uint64_t bar_storage;
+  __shared__ int abort_storage;
+  const uint32_t bar = tc::smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    tc::mbar_init(bar, 1);
+    abort_storage = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(status) != 0) return;   // poisoned by an earlier failure: do no work, as every kernel here
+  const tc::Abort ab{&abort_storage, status};
+  tc::mbar_wait(bar, 0, ab, where, limit_cycles);
+}
+}  // namespace
+
+cudaError_t launch_wait_selftest(int* status, long long limit_cycles, int where, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(status, limit_cycles, where);
+  return cudaGetLastError();
+}
+
 }  // namespace sp

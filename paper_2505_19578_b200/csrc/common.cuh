@@ -120,6 +120,9 @@ cudaError_t launch_determine_pattern(const PooledArgs& a, const float* pivot_row
 cudaError_t launch_last_row_distribution(const PooledArgs& a, float* out, cudaStream_t s);
 
 // bytes of per-tile softmax statistics the tensor-core kernel spills for one head
+// A one-warp kernel whose only wait cannot complete (host-visible check of the bounded-wait path).
+cudaError_t launch_wait_selftest(int* status, long long limit_cycles, int where, cudaStream_t s);
+
 inline size_t tile_stats_bytes_per_head(int Nb, int B) {
   return (size_t)Nb * (size_t)(Nb + 1) / 2 * (size_t)B * sizeof(float);
 }

@@ -46,7 +46,8 @@ struct Abort {
 // The checks are kept off the fast path: the CTA's own abort flag (shared memory) every 64
 // polls, the time limit and the global status word (a trip to L2 that would delay the wake-up
 // by hundreds of cycles if it were made often) every 4096.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where,
+                                          long long limit_cycles = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -60,7 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
         }
         const long long now = clock64();
         if (t0 == 0) t0 = now;
-        else if (now - t0 > kWaitCycles) break;
+        else if (now - t0 > limit_cycles) break;
       }
     }
   }
