@@ -42,8 +42,6 @@ from paper_2505_19578_b200 import synth  # noqa: E402
 # (profiles/attn_pair_kernel_llama8b_128k_dram_traffic.md); valid for the default workload, gamma and seed only,
 # and to be set back to None whenever the attention kernel changes.
 NCU_DRAM_TRAFFIC = {
-    ("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 1964069888 + 1183769600,
-    ("llama8b_128k", 131072, 0.9, 0, "block_sparse_attn"): 1487517952 + 900339968,
 }
 
 METRIC = "effective_tflops_prefill_attention_layer"

@@ -29,7 +29,18 @@
 // tiles then fall into step, their softmax phases coincide and nothing overlaps
 // the MMAs.)  P (bf16) overwrites the first half of the S columns it came from
 // and is the TMEM A operand of PV; the next QK of that tile is issued after the
-// PV that reads P, and the tensor pipe keeps issue order.
+// PV that reads P, and the tensor pipe keeps issue order.  The softmax finds the
+// row max of the whole tile first, so that P can be handed over in two halves:
+// the PV of keys 0..63 runs while keys 64..127 are still being exponentiated.
+//
+// Hand-offs.  Completion of MMAs and of TMA copies arrives on mbarriers
+// (tcgen05.commit, complete_tx).  What the issuing warp waits for comes through
+// named barriers instead: a poll of an mbarrier is a shared-memory round trip,
+// 150-250 cycles while the tensor pipe streams operands at the shared-memory
+// limit, and the issuing warp needs five or more hand-offs per key-block.  The
+// softmax warps `bar.arrive` when a half of P is stored, the producer warp
+// relays "K of the next key-block and V of this one have landed", the issuing
+// warp `bar.sync`s.
 //
 // Block importance in one pass: as in the single-tile kernel, each softmax
 // thread spills one float per visited tile, stat = m + log2(sum_c 2^(s_c - m))
@@ -38,7 +49,13 @@
 //
 // Every wait on an mbarrier is bounded: when it runs out the CTA raises an abort
 // flag, records SP_ERR_TIMEOUT in the status word, and all roles fall through
-// to the common teardown (TMEM is freed, the kernel returns).
+// to the common teardown (TMEM is freed, the kernel returns).  The named-barrier
+// syncs of the issuing warp have no limit of their own; they end because every
+// arrival they count is reached through bounded waits only, and is made also
+// when such a wait ran out (the warp that gave up arrives once more for the
+// step it was in, on ids taken in turn so that an early arrival never lands in
+// a phase the issuing warp has not left; the issuing warp looks at the abort
+// flag after the last sync of every key-block).
 #include "tc_ptx.cuh"
 
 namespace sp {
@@ -72,12 +89,17 @@ enum {
   BAR_V_FULL = BAR_K_EMPTY + kStages,
   BAR_V_EMPTY = BAR_V_FULL + kStages,
   BAR_S_FULL = BAR_V_EMPTY + kStages,  // + tile (A = 0, B = 1)
-  BAR_P_FULL = BAR_S_FULL + 2,
-  BAR_O_DONE = BAR_P_FULL + 2,
+  BAR_O_DONE = BAR_S_FULL + 2,
   BAR_COUNT = BAR_O_DONE + 2
 };
 
 enum { F_A = 1, F_B = 2, F_LAST = 4 };
+
+// Named barriers (0 is __syncthreads, 1 and 2 the epilogues of the two tiles): P of tile x ready (the four softmax
+// warps of the tile arrive, the issuing warp syncs), and K/V tiles of a merged key-block landed (the producer warp
+// arrives, the issuing warp syncs).  Ids are taken in turn — two per tile for P, four for K/V — so that an arrival
+// that comes early, e.g. the release after a wait ran out, never lands in a phase the other side has not left yet.
+enum { NB_P = 3, NB_KV = 11 };   // P: id NB_P + 4 * tile + 2 * half + (step & 1); K/V: id NB_KV + (key-block & 3)
 
 // ------------------------------------------------------------------ small PTX helpers of this kernel
 
@@ -229,7 +251,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(BAR_S_FULL + x), 1);
-      mbar_init(bar(BAR_P_FULL + x), 4);      // one arrival per softmax warp
       mbar_init(bar(BAR_O_DONE + x), 1);
     }
     *abort_flag = 0;
@@ -256,7 +277,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         const int cntA = tile[0].cnt, cntB = tile[1].cnt;
         const int32_t* idxA = tile[0].idx;
         const int32_t* idxB = tile[1].idx;
-        int pa = 0, pb = 0, n = 0, issued_k = 0, issued_v = 0;
+        int pa = 0, pb = 0, n = 0, issued_k = 0, issued_v = 0, relays = 0;
         int chunkA = 0, chunkB = 0;
         if (idxA) chunkA = lane < cntA ? idxA[lane] : 0;
         if (idxB) chunkB = lane < cntB ? idxB[lane] : 0;
@@ -277,7 +298,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           if (!(pa < cntA || pb < cntB)) f |= F_LAST;
           const int st = n % kStages;
           const uint32_t ph = (uint32_t)(n / kStages) & 1u;
-          if (n >= kStages) ok = mbar_wait(bar(BAR_K_EMPTY + st), ph ^ 1u, ab, 10);
+          if (n >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_K_EMPTY + st), ph ^ 1u, ab, 10));
           if (!ok) break;
           if (lane == 0) {
             kflags[st] = f;
@@ -286,7 +307,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
             trace(0, 20, n);
           }
           ++issued_k;
-          if (n >= kStages) ok = mbar_wait(bar(BAR_V_EMPTY + st), ph ^ 1u, ab, 11);
+          if (n >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_V_EMPTY + st), ph ^ 1u, ab, 11));
           if (!ok) break;
           if (lane == 0) {
             mbar_expect_tx(bar(BAR_V_FULL + st), kTile);
@@ -295,6 +316,25 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           }
           ++issued_v;
           ++n;
+          // relay for the issuing warp's iteration n - 2 (key-block n - 2 computed, n - 1 multiplied ahead):
+          // K of key-block n - 1 and V of key-block n - 2 have landed
+          if (n >= 2) {
+            const int mk = n - 1, mv = n - 2;
+            ok = mbar_wait(bar(BAR_K_FULL + mk % kStages), (uint32_t)(mk / kStages) & 1u, ab, 12);
+            if (ok) ok = mbar_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u, ab, 13);
+            ok = __all_sync(0xffffffffu, ok);
+            bar_arrive(NB_KV + (relays & 3), 64);     // also when a wait ran out: nobody may be left at a named barrier
+            ++relays;
+          }
+        }
+        if (__all_sync(0xffffffffu, ok) && n >= 1) {
+          // the last key-block: only its V is still awaited
+          const int mv = n - 1;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u, ab, 13));
+          bar_arrive(NB_KV + (relays & 3), 64);
+          ++relays;
+        } else if (n >= 1) {
+          bar_arrive(NB_KV + (relays & 3), 64);       // a wait ran out above: release the issuing warp once more
         }
         if (*abort_flag && lane == 0) {
           // let the copies already in flight land before the CTA gives its shared memory back
@@ -330,17 +370,18 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         mma_commit(bar(BAR_S_FULL + x));
       };
-      auto issue_pv = [&](int x, int st, bool accumulate) {   // O_x (+)= P_x V from V stage st
+      auto issue_pv = [&](int x, int st, int hf, bool accumulate) {   // O_x (+)= P_x V, keys 64 hf .. 64 hf + 63 of V stage st
         const uint64_t dv = dv0 + (uint64_t)((st * kTile) >> 4);
 #pragma unroll
-        for (int kk = 0; kk < BLK / 16; ++kk) {
-          // V tile: rows = keys (the MMA's K), 128-byte rows of 64 head-dim columns per box (N-major)
+        for (int k4 = 0; k4 < BLK / 32; ++k4) {
+          const int kk = hf * (BLK / 32) + k4;
           mma_ts(tmem + kOCol + x * 128, tmem + kSCol + x * 128 + kk * 8, dv + (uint32_t)((kk * 16 * 128) >> 4), idesc_pv,
                  (accumulate || kk > 0) ? 1u : 0u);
         }
       };
       bool ok = any_work ? mbar_wait(bar(BAR_Q_FULL), 0, ab, 20) : false;
       if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, ab, 21);
+      ok = __all_sync(0xffffffffu, ok);
       int f = 0, n = 0, tA = 0, tB = 0;
       if (ok) {
         tc_fence_after();
@@ -354,27 +395,31 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         __syncwarp();
       }
+      // The loop's hand-offs come through named barriers (a poll of an mbarrier costs the issuing warp 150-250
+      // cycles while the tensor pipe streams operands from shared memory; with five polls per key-block the
+      // warp was waiting a quarter of the time with nothing queued): the producer warp relays "K of the next
+      // key-block and V of this one have landed", the softmax warps "P of this tile is stored".  The flags of the
+      // next key-block and the abort flag are read from shared memory ahead of the MMAs whose issue hides the trip.
       while (ok) {
         const bool last = (f & F_LAST) != 0;
         const int st = n % kStages, stn = (n + 1) % kStages;
-        const uint32_t ph = (uint32_t)(n / kStages) & 1u, phn = (uint32_t)((n + 1) / kStages) & 1u;
-        int fn = 0;
-        if (!last) {
-          ok = mbar_wait(bar(BAR_K_FULL + stn), phn, ab, 22);
-          if (!ok) break;
-          fn = kflags[stn];
-        }
-        ok = mbar_wait(bar(BAR_V_FULL + st), ph, ab, 23);
-        if (!ok) break;
+        bar_sync(NB_KV + (n & 3), 64);
+        const int fn_early = last ? 0 : kflags[stn];
         if (f & F_A) {
-          ok = mbar_wait(bar(BAR_P_FULL + 0), tA & 1, ab, 24);
-          if (!ok) break;
+          bar_sync(NB_P + 0 + (tA & 1), 160);
+          tc_fence_after();
+          if (lane == 0) {
+            trace(1, 3, n);
+            issue_pv(0, st, 0, tA > 0);
+          }
+          __syncwarp();
+          bar_sync(NB_P + 2 + (tA & 1), 160);
         }
         tc_fence_after();
+        const int fn = fn_early;
         if (lane == 0) {
-          trace(1, 3, n);
           if (f & F_A) {
-            issue_pv(0, st, tA > 0);
+            issue_pv(0, st, 1, true);
             if (tA + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
           }
           if (fn & F_A) issue_qk(0, stn);
@@ -383,14 +428,20 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         __syncwarp();
         if (f & F_A) ++tA;
         if (f & F_B) {
-          ok = mbar_wait(bar(BAR_P_FULL + 1), tB & 1, ab, 25);
-          if (!ok) break;
+          bar_sync(NB_P + 4 + (tB & 1), 160);
+          tc_fence_after();
+          if (lane == 0) {
+            trace(1, 6, n);
+            issue_pv(1, st, 0, tB > 0);
+          }
+          __syncwarp();
+          bar_sync(NB_P + 6 + (tB & 1), 160);
         }
+        const int abort_raw = *abort_flag;       // after all syncs of this key-block; looked at after the MMAs below
         tc_fence_after();
         if (lane == 0) {
-          trace(1, 6, n);
           if (f & F_B) {
-            issue_pv(1, st, tB > 0);
+            issue_pv(1, st, 1, true);
             if (tB + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
           }
           mma_commit(bar(BAR_V_EMPTY + st));
@@ -400,7 +451,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         __syncwarp();
         if (f & F_B) ++tB;
-        if (last) break;
+        if (last || __any_sync(0xffffffffu, abort_raw != 0)) break;
         f = fn;
         ++n;
       }
@@ -425,23 +476,28 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     for (int t = 0; t < cnt && ok; ++t) {
       const int j = j_next;
       if (t + 1 < cnt) j_next = idx ? idx[t + 1] : t + 1;
-      ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, ab, 30 + x);
-      if (!ok) break;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + x), t & 1, ab, 30 + x));
+      if (!ok) {
+        bar_arrive(NB_P + 4 * x + 0 + (t & 1), 160);   // the issuing warp may be at this step's barriers: do not leave it there
+        bar_arrive(NB_P + 4 * x + 2 + (t & 1), 160);
+        break;
+      }
       tc_fence_after();
       if (tthread) trace(trole, 10, t);
-      // The 128 columns are taken as four chunks of 32, each an online-softmax step of its own:
-      // chunk max, (rarely) a move of the reference, exponentials, P chunk back into the columns
-      // that earlier chunks have already given up.  The next chunk's load is in flight meanwhile.
+      // Two sweeps over the 128 columns, 32 at a time with the next load in flight.  The first finds the row
+      // max and (rarely: only when it has grown by more than 2^8) moves the reference, rescaling O and the
+      // running sum; nothing of this key-block's P exists yet, so the PV of its first half may start while the
+      // second half is still being exponentiated.  The second sweep writes P (bf16) into columns the sweep
+      // has already given up and signals each half of the key-block as soon as it is stored.
       const bool diag = j == i;
-      float tile_sum = 0.f;
       uint32_t sa[32], sb[32];
       tmem_ld32_async(tS, sa);
-      auto chunk = [&](uint32_t* sc, const int c) {     // c: chunk index 0..3 (columns 32c .. 32c+31)
-        if (diag) {
+      auto mask_diag = [&](uint32_t* sc, const int c) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
-        }
+        for (int e = 0; e < 32; ++e)
+          if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
+      };
+      auto chunk_max = [&](const uint32_t* sc) {
         float mx0 = max3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
         float mx1 = max3(__uint_as_float(sc[3]), __uint_as_float(sc[4]), __uint_as_float(sc[5]));
         float mx2 = max3(__uint_as_float(sc[6]), __uint_as_float(sc[7]), __uint_as_float(sc[8]));
@@ -455,40 +511,51 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         mx0 = max3(mx0, __uint_as_float(sc[28]), __uint_as_float(sc[29]));
         mx1 = max3(mx1, __uint_as_float(sc[30]), __uint_as_float(sc[31]));
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale;
-        // the reference max only moves when the row max has grown by more than 2^8 (rare after the
-        // first chunk of the first key-block; a fully masked chunk has mx = -inf and leaves it alone)
-        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
-          const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
-          const float alpha = ex2_approx(m_ref - m_new);
-          if (t > 0) {
-            // O of the previous steps is relative to the old reference: bring it to the new one.
-            // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+        return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      };
+      float mx;
+      tmem_ld_wait();
+      reg_fence32(sa);
+      tmem_ld32_async(tS + 32, sb);
+      if (diag) mask_diag(sa, 0);
+      mx = chunk_max(sa);
+      tmem_ld_wait();
+      reg_fence32(sb);
+      tmem_ld32_async(tS + 64, sa);
+      if (diag) mask_diag(sb, 1);
+      mx = fmaxf(mx, chunk_max(sb));
+      tmem_ld_wait();
+      reg_fence32(sa);
+      tmem_ld32_async(tS + 96, sb);
+      if (diag) mask_diag(sa, 2);
+      mx = fmaxf(mx, chunk_max(sa));
+      tmem_ld_wait();
+      reg_fence32(sb);
+      tmem_ld32_async(tS, sa);                         // second sweep: chunk 0 again
+      if (diag) mask_diag(sb, 3);
+      mx = fmaxf(mx, chunk_max(sb)) * scale;
+      if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+        const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+        const float alpha = ex2_approx(m_ref - m_new);
+        if (t > 0) {
+          // O of the previous steps is relative to the old reference: bring it to the new one.
+          // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
 #pragma unroll 1
-            for (int oc = 0; oc < D / 32; ++oc) {
-              uint32_t o[32];
-              tmem_ld32(tO + oc * 32, o);
+          for (int oc = 0; oc < D / 32; ++oc) {
+            uint32_t o[32];
+            tmem_ld32(tO + oc * 32, o);
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st32(tO + oc * 32, o);
-            }
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tO + oc * 32, o);
           }
-          // the P chunks of this key-block that are already stored
-#pragma unroll 1
-          for (int pc = 0; pc < c; ++pc) {
-            uint32_t pp[16];
-            tmem_ld16(tS + pc * 16, pp);
-#pragma unroll
-            for (int e = 0; e < 16; ++e)
-              pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
-            tmem_st16(tS + pc * 16, pp);
-          }
-          l *= alpha;
-          tile_sum *= alpha;
-          m_ref = m_new;
         }
-        const float neg_m = -m_ref;
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        l *= alpha;
+        m_ref = m_new;
+      }
+      const float neg_m = -m_ref;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+      auto chunk = [&](uint32_t* sc, const int c) {     // c: chunk index 0..3 (columns 32c .. 32c+31)
+        if (diag) mask_diag(sc, c);
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
@@ -504,25 +571,31 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           pk[e / 2] = cvt_bf16x2(x0, x1);
           pk[e / 2 + 1] = cvt_bf16x2(x2, x3);
         }
-        tile_sum += (sum0 + sum1) + (sum2 + sum3);
         tmem_st16(tS + c * 16, pk);
       };
-#pragma unroll 1
-      for (int c = 0; c < 4; c += 2) {
-        tmem_ld_wait();
-        reg_fence32(sa);
-        tmem_ld32_async(tS + (c + 1) * 32, sb);
-        chunk(sa, c);
-        tmem_ld_wait();
-        reg_fence32(sb);
-        if (c == 0) tmem_ld32_async(tS + 64, sa);
-        chunk(sb, c + 1);
-      }
-      if (tthread) trace(trole, 13, t);
+      tmem_ld_wait();
+      reg_fence32(sa);
+      tmem_ld32_async(tS + 32, sb);
+      chunk(sa, 0);
+      tmem_ld_wait();
+      reg_fence32(sb);
+      tmem_ld32_async(tS + 64, sa);
+      chunk(sb, 1);
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_P_FULL + x));
+      bar_arrive(NB_P + 4 * x + 0 + (t & 1), 160);
+      if (tthread) trace(trole, 13, t);
+      tmem_ld_wait();
+      reg_fence32(sa);
+      tmem_ld32_async(tS + 96, sb);
+      chunk(sa, 2);
+      tmem_ld_wait();
+      reg_fence32(sb);
+      chunk(sb, 3);
+      tmem_wait_st();
+      tc_fence_before();
+      bar_arrive(NB_P + 4 * x + 2 + (t & 1), 160);
+      const float tile_sum = (sum0 + sum1) + (sum2 + sum3);
       if (tthread) trace(trole, 15, t);
       // off the critical path: running sum and the tile statistic
       l += tile_sum;

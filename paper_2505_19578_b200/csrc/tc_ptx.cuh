@@ -92,6 +92,15 @@ __device__ __forceinline__ bool bar_and(int id, int threads, bool pred) {
   return out != 0;
 }
 
+// Named barriers as a hand-off that does not go through shared memory (an mbarrier poll is a shared-memory round
+// trip, slow while the tensor pipe streams operands): the producer side arrives, the consumer side syncs.
+__device__ __forceinline__ void bar_arrive(int id, int threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
