@@ -484,12 +484,14 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       }
       tc_fence_after();
       if (tthread) trace(trole, 10, t);
-      // Two sweeps over the 128 columns, 32 at a time with the next load in flight.  The first finds the row
-      // max and (rarely: only when it has grown by more than 2^8) moves the reference, rescaling O and the
-      // running sum; nothing of this key-block's P exists yet, so the PV of its first half may start while the
-      // second half is still being exponentiated.  The second sweep writes P (bf16) into columns the sweep
-      // has already given up and signals each half of the key-block as soon as it is stored.
+      // The 128 columns are taken as four chunks of 32 (`tcgen05.ld.32x32b.x32`, the next chunk's load in flight).
+      // Chunks 0 and 1 are online-softmax steps of their own: chunk max, (rarely: only when the row max has grown
+      // by more than 2^8) a move of the reference, exponentials, P chunk into columns the sweep has given up.
+      // Then the max of chunks 2 and 3 is taken, and a move they ask for is made, BEFORE the first half of P is
+      // handed over: after that no reference can move in this key-block, so the PV of keys 0..63 may run while
+      // keys 64..127 are exponentiated from the registers they already sit in.
       const bool diag = j == i;
+      float tile_sum = 0.f;
       uint32_t sa[32], sb[32];
       tmem_ld32_async(tS, sa);
       auto mask_diag = [&](uint32_t* sc, const int c) {
@@ -513,49 +515,43 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         mx1 = max3(mx1, __uint_as_float(sc[30]), __uint_as_float(sc[31]));
         return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       };
-      float mx;
-      tmem_ld_wait();
-      reg_fence32(sa);
-      tmem_ld32_async(tS + 32, sb);
-      if (diag) mask_diag(sa, 0);
-      mx = chunk_max(sa);
-      tmem_ld_wait();
-      reg_fence32(sb);
-      tmem_ld32_async(tS + 64, sa);
-      if (diag) mask_diag(sb, 1);
-      mx = fmaxf(mx, chunk_max(sb));
-      tmem_ld_wait();
-      reg_fence32(sa);
-      tmem_ld32_async(tS + 96, sb);
-      if (diag) mask_diag(sa, 2);
-      mx = fmaxf(mx, chunk_max(sa));
-      tmem_ld_wait();
-      reg_fence32(sb);
-      tmem_ld32_async(tS, sa);                         // second sweep: chunk 0 again
-      if (diag) mask_diag(sb, 3);
-      mx = fmaxf(mx, chunk_max(sb)) * scale;
-      if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
-        const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
-        const float alpha = ex2_approx(m_ref - m_new);
-        if (t > 0) {
-          // O of the previous steps is relative to the old reference: bring it to the new one.
-          // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+      // mx: scaled max of the columns about to be exponentiated; stored: P chunks of this key-block already in TMEM
+      auto move_reference = [&](const float mx, const int stored) {
+        // the reference max only moves when the row max has grown by more than 2^8 (rare after the first chunk of
+        // the first key-block; a fully masked chunk has mx = -inf and leaves it alone)
+        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+          const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+          const float alpha = ex2_approx(m_ref - m_new);
+          if (t > 0) {
+            // O of the previous steps is relative to the old reference: bring it to the new one.
+            // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
 #pragma unroll 1
-          for (int oc = 0; oc < D / 32; ++oc) {
-            uint32_t o[32];
-            tmem_ld32(tO + oc * 32, o);
+            for (int oc = 0; oc < D / 32; ++oc) {
+              uint32_t o[32];
+              tmem_ld32(tO + oc * 32, o);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tO + oc * 32, o);
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+              tmem_st32(tO + oc * 32, o);
+            }
           }
+          // the P chunks of this key-block that are already stored (none of them handed over yet)
+#pragma unroll 1
+          for (int pc = 0; pc < stored; ++pc) {
+            uint32_t pp[16];
+            tmem_ld16(tS + pc * 16, pp);
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+              pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
+            tmem_st16(tS + pc * 16, pp);
+          }
+          l *= alpha;
+          tile_sum *= alpha;
+          m_ref = m_new;
         }
-        l *= alpha;
-        m_ref = m_new;
-      }
-      const float neg_m = -m_ref;
-      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-      auto chunk = [&](uint32_t* sc, const int c) {     // c: chunk index 0..3 (columns 32c .. 32c+31)
-        if (diag) mask_diag(sc, c);
+      };
+      auto chunk_exps = [&](const uint32_t* sc, const int c) {   // exponentials, sums, P chunk c (columns 32c .. 32c+31)
+        const float neg_m = -m_ref;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
@@ -571,31 +567,40 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           pk[e / 2] = cvt_bf16x2(x0, x1);
           pk[e / 2 + 1] = cvt_bf16x2(x2, x3);
         }
+        tile_sum += (sum0 + sum1) + (sum2 + sum3);
         tmem_st16(tS + c * 16, pk);
       };
       tmem_ld_wait();
       reg_fence32(sa);
       tmem_ld32_async(tS + 32, sb);
-      chunk(sa, 0);
+      if (diag) mask_diag(sa, 0);
+      move_reference(chunk_max(sa) * scale, 0);
+      chunk_exps(sa, 0);
       tmem_ld_wait();
       reg_fence32(sb);
       tmem_ld32_async(tS + 64, sa);
-      chunk(sb, 1);
+      if (diag) mask_diag(sb, 1);
+      move_reference(chunk_max(sb) * scale, 1);
+      chunk_exps(sb, 1);
+      tmem_ld_wait();
+      reg_fence32(sa);
+      tmem_ld32_async(tS + 96, sb);
+      if (diag) mask_diag(sa, 2);
+      float mx23 = chunk_max(sa);
+      tmem_ld_wait();
+      reg_fence32(sb);
+      if (diag) mask_diag(sb, 3);
+      mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
+      move_reference(mx23, 2);
       tmem_wait_st();
       tc_fence_before();
       bar_arrive(NB_P + 4 * x + 0 + (t & 1), 160);
       if (tthread) trace(trole, 13, t);
-      tmem_ld_wait();
-      reg_fence32(sa);
-      tmem_ld32_async(tS + 96, sb);
-      chunk(sa, 2);
-      tmem_ld_wait();
-      reg_fence32(sb);
-      chunk(sb, 3);
+      chunk_exps(sa, 2);
+      chunk_exps(sb, 3);
       tmem_wait_st();
       tc_fence_before();
       bar_arrive(NB_P + 4 * x + 2 + (t & 1), 160);
-      const float tile_sum = (sum0 + sum1) + (sum2 + sum3);
       if (tthread) trace(trole, 15, t);
       // off the critical path: running sum and the tile statistic
       l += tile_sum;
