@@ -398,8 +398,10 @@ int sp_ctx_set_kernel(sp_ctx* ctx, int which);
  * pairs {(event_id << 32) | step, SM clock} into
  * events[(role * events_per_role + n) * 2 .. +1].  Event ids: 20/21 K/V load
  * issued; 1 K tile landed, 2 QK^T issued, 3 P and V ready, 4 PV issued; 10 S
- * ready, 11 S in registers, 12 row max done, 13 exponentials done, 14 O
- * rescaled, 15 P stored and signalled.  `events` is a device buffer of
+ * ready, 11 S in registers, 12 row max done, 13 exponentials done (paired
+ * kernel: first half of P handed over), 14 O rescaled, 15 P stored and
+ * signalled; paired kernel, issuer: 3/5 around the MMAs of the first
+ * row-block, 6/4 around those of the second.  `events` is a device buffer of
  * 5 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
  * switches tracing off. */
 int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
