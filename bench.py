@@ -42,8 +42,8 @@ from paper_2505_19578_b200 import synth  # noqa: E402
 # (profiles/attn_pair_kernel_llama8b_128k_dram_traffic.md); valid for the default workload, gamma and seed only,
 # and to be set back to None whenever the attention kernel changes.
 NCU_DRAM_TRAFFIC = {
-    ("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 1969306624 + 1190285568,
-    ("llama8b_128k", 131072, 0.9, 0, "block_sparse_attn"): 1488921856 + 904208128,
+    ("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 1970131456 + 1190532096,
+    ("llama8b_128k", 131072, 0.9, 0, "block_sparse_attn"): 1485898496 + 903549440,
 }
 
 METRIC = "effective_tflops_prefill_attention_layer"

@@ -152,21 +152,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
-// (d0, d1) = (a0, a1) * (b, b) + (c, c): one packed FMA
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
-  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
-      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b), "f"(c));
-}
-__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
-  asm("{\n\t.reg .b64 ra, rd;\n\t"
-      "mov.b64 rd, {%0, %1};\n\tmov.b64 ra, {%2, %3};\n\t"
-      "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "+f"(d0), "+f"(d1)
-      : "f"(a0), "f"(a1));
-}
 // bf16x2 with `lo` in the low half
 __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
   uint32_t d;
@@ -550,24 +535,23 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
       };
       auto chunk_exps = [&](const uint32_t* sc, const int c) {   // exponentials, sums, P chunk c (columns 32c .. 32c+31)
-        const float neg_m = -m_ref;
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_ref, -m_ref);
+        float2 sum01 = make_float2(0.f, 0.f), sum23 = make_float2(0.f, 0.f);
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
-          float x0, x1, x2, x3;
-          fma2(x0, x1, __uint_as_float(sc[e]), __uint_as_float(sc[e + 1]), scale, neg_m);
-          fma2(x2, x3, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]), scale, neg_m);
-          x0 = ex2_approx(x0);
-          x1 = ex2_approx(x1);
-          x2 = ex2_approx(x2);
-          x3 = ex2_approx(x3);
-          add2(sum0, sum1, x0, x1);
-          add2(sum2, sum3, x2, x3);
-          pk[e / 2] = cvt_bf16x2(x0, x1);
-          pk[e / 2 + 1] = cvt_bf16x2(x2, x3);
+          float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sc[e]), __uint_as_float(sc[e + 1])), sc2, nm2);
+          float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3])), sc2, nm2);
+          x01.x = ex2_approx(x01.x);
+          x01.y = ex2_approx(x01.y);
+          x23.x = ex2_approx(x23.x);
+          x23.y = ex2_approx(x23.y);
+          sum01 = __fadd2_rn(sum01, x01);
+          sum23 = __fadd2_rn(sum23, x23);
+          pk[e / 2] = cvt_bf16x2(x01.x, x01.y);
+          pk[e / 2 + 1] = cvt_bf16x2(x23.x, x23.y);
         }
-        tile_sum += (sum0 + sum1) + (sum2 + sum3);
+        tile_sum += (sum01.x + sum01.y) + (sum23.x + sum23.y);
         tmem_st16(tS + c * 16, pk);
       };
       tmem_ld_wait();
