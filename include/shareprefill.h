@@ -78,7 +78,16 @@ int sp_ctx_create(sp_ctx** out, int device);
 int sp_ctx_destroy(sp_ctx* ctx);
 
 /* Bytes of workspace sp_prefill_attn needs for a problem of this size
- * (importance maps, masks, compacted lists, per-tile softmax statistics). */
+ * (importance maps, masks, compacted lists, per-tile softmax statistics; the
+ * statistics are sized for the SM count of the current CUDA device).
+ *
+ * Which calls may allocate: any call that takes a context grows the context's
+ * workspace when the problem needs more than it holds (cudaDeviceSynchronize,
+ * cudaFree, cudaMalloc: it synchronises the device that one time), and
+ * sp_prefill_attn_host does the same for its device copies of q, k, v and out.
+ * Reserve ahead (sp_ctx_reserve) to keep the calls free of both: the figure
+ * returned here covers sp_prefill_attn, sp_dense_pivot_attn,
+ * sp_block_sparse_attn and the workspace part of sp_prefill_attn_host. */
 int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block,
                        int n_pivots, size_t* bytes /* host, out */);
 
@@ -141,27 +150,37 @@ int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, con
  *   no allocating library routine.
  *
  *   Same arguments and results as sp_dense_pivot_attn, plus `device`, the CUDA
- *   device the tensors live on.  Limits and rules:
- *   - with importance_out != NULL the launch needs
- *     n_heads * Nb * (Nb + 1) / 2 * block * 4 bytes of statistics; beyond 64 MiB the
- *     call returns SP_ERR_SCRATCH_LIMIT and launches nothing (e.g. seq 16384, block
- *     128: 15 heads per call; seq 32768: 3 heads).  Without importance no scratch
- *     is used and there is no limit.
+ *   device the tensors live on, and the same kernels: at head_dim 128 and block 128
+ *   the persistent kernel that gives a CTA two adjacent row-blocks, otherwise the
+ *   one-row-block kernel.  Limits and rules:
+ *   - with importance_out != NULL the launch needs statistics scratch: at head_dim
+ *     128 / block 128, min(SMs of the device, n_heads * ceil(Nb / 2)) * 2 * Nb * 128 * 4
+ *     bytes (148 SMs: any number of heads up to seq 56576); for the other shapes
+ *     n_heads * Nb * (Nb + 1) / 2 * block * 4 bytes.  Beyond 64 MiB the call returns
+ *     SP_ERR_SCRATCH_LIMIT and launches nothing.  Without importance no scratch is
+ *     used and there is no limit.
  *   - the first call on a device looks up the array's device address (a host-side
- *     query, done with that device current).  Make that first call outside any
+ *     query, done with that device current).  With lazy module loading that query is
+ *     also what loads the array's module, i.e. the moment the 64 MiB are taken from
+ *     the device: it can synchronise, and on a device whose memory is already all in
+ *     use it fails (SP_ERR_CUDA).  Make that first call at start-up, outside any
  *     stream capture.
- *   - all calls on a device share the one array and one status word.  The array
- *     keeps whatever the last call left in it; nothing in it needs to start at
- *     zero, and the status word is cleared on the stream before every launch.
- *     Two calls whose kernels may run at the same time on the same device
- *     (different streams, or different host threads) race on it: serialise them.
+ *   - all calls on a device share the one array, one status word and one work
+ *     counter.  The array keeps whatever the last call left in it; nothing in it
+ *     needs to start at zero, and status word and counter are cleared on the stream
+ *     before every launch.  Two calls whose kernels may run at the same time on the
+ *     same device (different streams, or different host threads) race on them:
+ *     serialise them.
  *   - a device-side wait that runs out makes the kernel stop early, as in the
- *     context version, but this variant has no call to read the status word back.
+ *     context version: outputs are then incomplete.  sp_fixed_scratch_status reads
+ *     that status word (after the caller has synchronised): *code is SP_OK or
+ *     SP_ERR_TIMEOUT.  It allocates nothing either.
  */
 #define SP_FIXED_SCRATCH_BYTES (64ull << 20)
 int sp_dense_pivot_attn_fixed_scratch(int device, const sp_tensor* q, const sp_tensor* k, const sp_tensor* v,
                                       const int32_t* heads, int n_heads, int block, sp_tensor* out,
                                       float* importance_out, float* lse_out, void* stream);
+int sp_fixed_scratch_status(int device, int* code /* host, out */, int* where /* host, out */);
 
 /*
  * Step 2 - importance map -> block mask and compacted key-block lists.
@@ -380,35 +399,6 @@ int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q
                           const sp_tensor* v, const int32_t* cluster_of_head, float gamma, float delta,
                           float tau, int block, int pooled_construction, sp_tensor* out,
                           uint8_t* mask_out, int32_t* pattern_out, void* stream);
-
-/* Which attention kernel the context launches: 0 = tensor-core kernels
- * (tcgen05 / TMEM / TMA; the product path, default: for head_dim 128 and block
- * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V
- * tiles, otherwise the one-row-block kernel), 1 = plain fp32 CUDA-core kernel
- * kept as an independent on-device cross-check, 2 = the one-row-block
- * tensor-core kernel for every shape. */
-int sp_ctx_set_kernel(sp_ctx* ctx, int which);
-
-/* Phase trace of the tensor-core attention kernels (a profiling aid).  While a
- * buffer is set, the CTA that owns the longest row-block(s) of the first listed
- * head of every attention launch records, for each of its roles (0 = TMA
- * producer, 1 = MMA issuer (of the first row-block), 2 = softmax thread 0 of the
- * first row-block; paired kernel only: 3 = softmax thread 0 of the second
- * row-block, 4 = its MMA issuer), up to `events_per_role`
- * pairs {(event_id << 32) | step, SM clock} into
- * events[(role * events_per_role + n) * 2 .. +1].  Event ids: 20/21 K/V load
- * issued; 1 K tile landed, 2 QK^T issued, 3 P and V ready, 4 PV issued; 10 S
- * ready, 11 S in registers, 12 row max done, 13 exponentials done (paired
- * kernel: first half of P handed over), 14 O rescaled, 15 P stored and
- * signalled; paired kernel, issuer: 3/5 around the MMAs of the first
- * row-block, 6/4 around those of the second.  `events` is a device buffer of
- * 5 * events_per_role * 2 int64 that the caller zeroes; events_per_role = 0
- * switches tracing off. */
-int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
-
-/* Number of kernels this context has launched since creation (for callers
- * that account for launches). */
-int64_t sp_ctx_launch_count(const sp_ctx* ctx);
 
 #ifdef __cplusplus
 }

@@ -32,7 +32,7 @@ EXPORTS = (
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
     "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
     "sp_dict_create", "sp_dict_destroy", "sp_dict_clear", "sp_dict_count", "sp_prefill_attn_layer",
-    "sp_selftest_wait_timeout",
+    "sp_selftest_wait_timeout", "sp_fixed_scratch_status",
 )
 
 
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
     lib.sp_strerror.restype = ctypes.c_char_p
     lib.sp_dense_pivot_attn.argtypes = [P, T, T, T, IP, I, I, T, P, P, P]
     lib.sp_dense_pivot_attn_fixed_scratch.argtypes = [I, T, T, T, IP, I, I, T, P, P, P]
+    lib.sp_fixed_scratch_status.argtypes = [I, IP, IP]
     lib.sp_block_mask_from_importance.argtypes = [P, P, I, I, F, P, P, P, P]
     lib.sp_block_sparse_attn.argtypes = [P, T, T, T, IP, I, IP, P, P, I, I, T, P]
     lib.sp_prefill_attn.argtypes = [P, T, T, T, IP, IP, I, F, I, T, P, P]
@@ -313,6 +314,15 @@ def sp_dense_pivot_attn_fixed_scratch(q, k, v, heads, block, out, importance_out
     _check(load().sp_dense_pivot_attn_fixed_scratch(dev, _view(q), _view(k), _view(v), _i32(heads), len(heads), block,
                                                     _view(out), _ptr(importance_out), _ptr(lse_out), _stream(stream)),
            "sp_dense_pivot_attn_fixed_scratch")
+
+
+def fixed_scratch_status(device=0):
+    """(code, where) of the allocation-free entry point's status word on `device`; clears it when set.
+
+    Synchronise the stream the call was made on first."""
+    code, where = ctypes.c_int(), ctypes.c_int()
+    _check(load().sp_fixed_scratch_status(int(device), ctypes.byref(code), ctypes.byref(where)), "sp_fixed_scratch_status")
+    return code.value, where.value
 
 
 def workspace_bytes(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots) -> int:

@@ -14,7 +14,7 @@ struct sp_ctx {
   int device = 0;
   void* ws = nullptr;
   size_t ws_bytes = 0;
-  int* status = nullptr;  // device int[2]
+  int* status = nullptr;  // device int[4]: {code, where, work counter of the paired kernel, unused}
   int kernel = 0;         // 0 tensor-core (paired where supported), 1 CUDA-core cross-check, 2 tensor-core single-tile
   int64_t launches = 0;
   long long* trace = nullptr;  // caller's device buffer for the phase trace, or null
@@ -72,6 +72,10 @@ int check_tensor(const sp_tensor* t) {
   if ((reinterpret_cast<uintptr_t>(t->data) & 15) != 0) return SP_ERR_INVALID_ARG;
   for (int x = 0; x < 3; ++x)
     if (t->stride[x] < 0 || (t->stride[x] % 8) != 0) return SP_ERR_INVALID_ARG;
+  // a broadcast view (stride 0 over heads or rows, e.g. an expanded K) would make the tensor maps address memory
+  // past the caller's buffer: refuse it
+  for (int x = 1; x < 3; ++x)
+    if (t->stride[x] == 0 && t->shape[x] > 1) return SP_ERR_INVALID_ARG;
   if (t->stride[2] < t->shape[3]) return SP_ERR_INVALID_ARG;
   return SP_OK;
 }
@@ -113,6 +117,7 @@ AttnArgs base_args(const sp_ctx* ctx, const Problem& p, const sp_tensor* q, cons
   a.n_q_heads = p.Hq; a.n_kv_heads = p.Hkv;
   a.N = p.N; a.d = p.d; a.B = p.B; a.Nb = p.Nb; a.group = p.Hq / p.Hkv;
   a.status = ctx->status;
+  a.work_counter = ctx->status ? ctx->status + 2 : nullptr;
   a.trace = ctx->trace;
   a.trace_cap = ctx->trace_cap;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.d));
@@ -148,11 +153,18 @@ int launch_attn(sp_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   return SP_OK;
 }
 
+// Bytes of tile statistics a dense launch over n_heads heads with importance needs.  `paired`: the launch goes to the
+// paired kernel (one region per CTA, used by every launch in turn); otherwise one region per head.
+bool goes_paired(int kernel, int d, int B) { return kernel == 0 && d == 128 && B == 128; }
+size_t stats_bytes(bool paired, int n_heads, int Nb, int B) {
+  return paired ? attn_pair_stats_bytes(n_heads, Nb) : (size_t)n_heads * tile_stats_bytes_per_head(Nb, B);
+}
+
 struct WsLayout {
   size_t imp, mask, counts, indices, stats, total;
 };
 
-WsLayout ws_layout(int Nb, int B, int n_pivots) {
+WsLayout ws_layout(int Nb, int B, int n_pivots, bool paired) {
   WsLayout w;
   size_t off = 0;
   const size_t nn = (size_t)Nb * Nb;
@@ -160,7 +172,7 @@ WsLayout ws_layout(int Nb, int B, int n_pivots) {
   w.mask = off;    off += align_up(n_pivots * nn);
   w.counts = off;  off += align_up((size_t)n_pivots * Nb * sizeof(int32_t));
   w.indices = off; off += align_up(n_pivots * nn * sizeof(int32_t));
-  w.stats = off;   off += align_up(n_pivots * tile_stats_bytes_per_head(Nb, B));
+  w.stats = off;   off += align_up(stats_bytes(paired, n_pivots, Nb, B));
   w.total = off;
   return w;
 }
@@ -206,7 +218,7 @@ int sp_ctx_create(sp_ctx** out, int device) {
   sp_ctx* c = new (std::nothrow) sp_ctx();
   if (!c) return SP_ERR_WORKSPACE;
   c->device = device;
-  if (cudaMalloc(&c->status, 2 * sizeof(int)) != cudaSuccess || cudaMemset(c->status, 0, 2 * sizeof(int)) != cudaSuccess) {
+  if (cudaMalloc(&c->status, 4 * sizeof(int)) != cudaSuccess || cudaMemset(c->status, 0, 4 * sizeof(int)) != cudaSuccess) {
     cudaGetLastError();
     delete c;
     return SP_ERR_CUDA;
@@ -234,7 +246,7 @@ int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim,
   if (block != 64 && block != 128) return SP_ERR_UNSUPPORTED;
   if (head_dim != 64 && head_dim != 128) return SP_ERR_UNSUPPORTED;
   if (seq % block != 0 || seq / block > kMaxNb || n_q_heads % n_kv_heads != 0) return SP_ERR_UNSUPPORTED;
-  *bytes = ws_layout((int)(seq / block), block, n_pivots).total;
+  *bytes = ws_layout((int)(seq / block), block, n_pivots, goes_paired(0, head_dim, block)).total;
   return SP_OK;
 }
 
@@ -300,7 +312,7 @@ int sp_dense_pivot_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, con
   a.importance = importance_out;
   a.lse = lse_out;
   if (importance_out && ctx->kernel != 1) {
-    if ((rc = reserve(ctx, align_up((size_t)n_heads * tile_stats_bytes_per_head(p.Nb, p.B))))) return rc;
+    if ((rc = reserve(ctx, align_up(stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_heads, p.Nb, p.B))))) return rc;
     a.tile_stats = static_cast<float*>(ctx->ws);
   }
   return launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
@@ -316,8 +328,6 @@ int sp_dense_pivot_attn_fixed_scratch(int device, const sp_tensor* q, const sp_t
   if (n_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
   for (int t = 0; t < n_heads; ++t)
     if (heads[t] < 0 || heads[t] >= p.Hq) return SP_ERR_INVALID_ARG;
-  if (importance_out && (size_t)n_heads * tile_stats_bytes_per_head(p.Nb, p.B) > kFixedScratchBytes)
-    return SP_ERR_SCRATCH_LIMIT;
   if (n_heads == 0) return SP_OK;
   DeviceGuard g(device);
   if (!g.ok) return SP_ERR_CUDA;
@@ -327,7 +337,15 @@ int sp_dense_pivot_attn_fixed_scratch(int device, const sp_tensor* q, const sp_t
   for (int t = 0; t < n_heads; ++t) { a.heads.v[t] = heads[t]; a.lists.v[t] = -1; }
   a.importance = importance_out;
   a.lse = lse_out;
-  if (launch_attn_tc_fixed_scratch(a, device, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  if (fixed_scratch_need(a) > kFixedScratchBytes) return SP_ERR_SCRATCH_LIMIT;
+  if (launch_attn_fixed_scratch(a, device, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SP_ERR_CUDA;
+  return SP_OK;
+}
+
+int sp_fixed_scratch_status(int device, int* code, int* where) {
+  DeviceGuard g(device);
+  if (!g.ok) return SP_ERR_CUDA;
+  if (fixed_status_read(device, code, where) != cudaSuccess) { cudaGetLastError(); return SP_ERR_CUDA; }
   return SP_OK;
 }
 
@@ -399,7 +417,7 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
   DeviceGuard g(ctx->device);
   if (!g.ok) return SP_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots);
+  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots, goes_paired(ctx->kernel, p.d, p.B));
   if ((rc = reserve(ctx, w.total))) return rc;
   char* ws = static_cast<char*>(ctx->ws);
   float* imp = reinterpret_cast<float*>(ws + w.imp);
@@ -528,7 +546,8 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
   Problem p;
   int rc = check_problem(&q, &k, &v, &o, block, &p);
   if (rc) return rc;
-  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots);
+  const bool paired = goes_paired(ctx->kernel, p.d, p.B);
+  const WsLayout w = ws_layout(p.Nb, p.B, n_pivots, paired);
   if ((rc = reserve(ctx, w.total))) return rc;
   char* ws = static_cast<char*>(ctx->ws);
   float* imp = reinterpret_cast<float*>(ws + w.imp);
@@ -587,7 +606,7 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
       a.n_heads = u1 - u0;
       for (int t = u0; t < u1; ++t) { a.heads.v[t - u0] = pivot_heads[t]; a.lists.v[t - u0] = -1; }
       a.importance = imp + (size_t)u0 * nn;
-      a.tile_stats = stats + (size_t)u0 * stats_floats_per_head;
+      a.tile_stats = paired ? stats : stats + (size_t)u0 * stats_floats_per_head;   // launches on one stream take turns
       if (int r = launch_attn(ctx, a, sc)) return r;
       if (!hand_over(sc, sout)) return SP_ERR_CUDA;
       for (int t = u0; t < u1; ++t)
@@ -829,7 +848,7 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   const size_t o_counts = take((size_t)n_lists * p.Nb * sizeof(int32_t));
   const size_t o_indices = take(n_lists * nn * sizeof(int32_t));
   const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_pivots, p.Nb, p.d) * sizeof(float)
-                                                    : (size_t)n_pivots * tile_stats_bytes_per_head(p.Nb, p.B));
+                                                    : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_pivots, p.Nb, p.B));
   const size_t o_atilde = take((size_t)n_pivots * p.Nb * sizeof(float));
   const size_t o_rows = take((size_t)n_row * p.Nb * sizeof(float));
   const size_t o_small = take((size_t)(3 * kMaxHeads + p.Hq) * sizeof(int32_t));
@@ -1011,7 +1030,7 @@ int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q
   const size_t o_imp = take(n_new_max * nn * sizeof(float));
   const size_t o_scores = take(pooled_construction ? nn * sizeof(float) : 0);
   const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_new_max, p.Nb, p.d) * sizeof(float)
-                                                    : (size_t)n_new_max * tile_stats_bytes_per_head(p.Nb, p.B));
+                                                    : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_new_max, p.Nb, p.B));
   const size_t o_vs = take(vslash_scratch_bytes(p.Hq, p.N, 8));
   if ((rc = reserve(ctx, off))) return rc;
   char* ws = static_cast<char*>(ctx->ws);

@@ -6,21 +6,31 @@
 //   probability mass of each (query-block, key-block) tile; a member walks the
 //   compacted list of key-blocks its cluster's pivot selected.
 //
-// One CTA owns one head and TWO adjacent query row-blocks (tile A = row-block
-// 2u, tile B = row-block 2u+1), 256 query rows, and occupies a whole SM.  The
-// two tiles walk the UNION of their key-block lists in ascending order, so a
-// K/V tile both of them need is brought into shared memory once and feeds four
-// MMAs instead of two; a key-block only one of them selected is computed for
-// that tile alone.  (Dense: the union is 0..2u+1, the last key-block is B's
-// diagonal tile only.)
+// Persistent CTAs, one per SM.  A work item is one head and TWO adjacent query
+// row-blocks (tile A = row-block 2u, tile B = row-block 2u+1), 256 query rows.
+// The items of a launch are ordered (the heads of one KV head together, the
+// longest pairs first) and handed out through a device counter, so an SM that
+// finishes early takes the next item; barriers and tensor memory are set up once
+// per CTA, and the loads and the first QK^T of the next item are issued while the
+// softmax warps still write out the item before.  The two tiles walk the UNION
+// of their key-block lists in ascending order, so a K/V tile both of them need
+// is brought into shared memory once and feeds four MMAs instead of two; a
+// key-block only one of them selected is computed for that tile alone.  (Dense:
+// the union is 0..2u+1, the last key-block is B's diagonal tile only.)
 //
-// Warp roles (320 threads):
+// Warp roles (352 threads):
 //   warps 0-3   softmax of tile A: thread t owns query row t = TMEM lane t
 //   warps 4-7   softmax of tile B
 //   warp  8     MMA issuer, owner of the TMEM allocation (all 512 columns:
 //               S_A, S_B, O_A, O_B, 128 fp32 columns each)
-//   warp  9     producer: merges the two lists, TMA loads of Q (once) and of
-//               the K and V tiles into two-stage rings (128-byte swizzle)
+//   warp  9     producer: merges the two lists, TMA loads of Q (once per item)
+//               and of the K and V tiles into two-stage rings (128-byte swizzle)
+//   warp 10     scheduler: takes the next item from the counter, resolves it to
+//               (head, pair, list, counts) and posts it, one item ahead, in a
+//               two-slot ring of shared memory that the other ten warps read
+//
+// Rings, barrier phases and named-barrier ids run on across items (every role
+// counts key-blocks, tile steps and items for itself).
 //
 // Order of the MMAs, per merged key-block n:  PV_A(n), QK_A(n+1), PV_B(n),
 // QK_B(n+1), all issued by one thread: while the softmax warps of A work on
@@ -46,6 +56,8 @@
 // thread spills one float per visited tile, stat = m + log2(sum_c 2^(s_c - m))
 // with m the row's reference max at that step; after the last tile the row's
 // log-sum-exp L is known and the tile mass is (1/B) sum_rows 2^(stat - L).
+// The statistics of an item live only until its epilogue, so each CTA owns one
+// region of 2 * Nb * B floats that every item it runs writes and reads in turn.
 //
 // Every wait on an mbarrier is bounded: when it runs out the CTA raises an abort
 // flag, records SP_ERR_TIMEOUT in the status word, and all roles fall through
@@ -65,7 +77,8 @@ using namespace tc;
 
 constexpr int D = 128;      // head_dim
 constexpr int BLK = 128;    // block
-constexpr int kThreadsPair = 320;
+constexpr int kThreadsPair = 352;   // eight softmax warps, the issuing, the producer and the scheduler warp
+constexpr int kItemReaders = 10;     // warps that take every work item: all but the scheduler
 constexpr int kStages = 2;  // K ring and V ring depth
 
 // shared-memory plan (bytes)
@@ -84,14 +97,18 @@ constexpr uint32_t kOCol = 256;    // O_A at 256, O_B at 384
 
 enum {
   BAR_Q_FULL = 0,
+  BAR_Q_EMPTY,
   BAR_K_FULL,                          // + stage
   BAR_K_EMPTY = BAR_K_FULL + kStages,  // + stage
   BAR_V_FULL = BAR_K_EMPTY + kStages,
   BAR_V_EMPTY = BAR_V_FULL + kStages,
   BAR_S_FULL = BAR_V_EMPTY + kStages,  // + tile (A = 0, B = 1)
   BAR_O_DONE = BAR_S_FULL + 2,
-  BAR_COUNT = BAR_O_DONE + 2
+  BAR_ITEM_FULL = BAR_O_DONE + 2,      // + item slot
+  BAR_ITEM_EMPTY = BAR_ITEM_FULL + 2,
+  BAR_COUNT = BAR_ITEM_EMPTY + 2
 };
+static_assert(BAR_COUNT * 8 <= 256, "barriers overlap the TMEM slot");
 
 enum { F_A = 1, F_B = 2, F_LAST = 4 };
 
@@ -159,11 +176,15 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
   return d;
 }
 
-// One tile's geometry as seen by every role.
-struct TileInfo {
-  int i;                 // row-block
-  int cnt;               // key-blocks it visits
-  const int32_t* idx;    // its ascending key-block list, or null = 0..i
+// One work item as the scheduler warp posts it to the other roles (shared memory, two slots of eight ints).
+struct Item {
+  int id;      // position in the work order, -1 = no more work
+  int slot;    // position of the head in the call's head table
+  int u;       // pair of row-blocks 2u, 2u + 1
+  int h;       // query head
+  int list;    // list index, -1 = dense
+  int cntA;    // key-blocks tile A visits
+  int cntB;    // key-blocks tile B visits
 };
 
 __global__ void __launch_bounds__(kThreadsPair, 1)
@@ -177,42 +198,11 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kMiscOff + 260);
   volatile int* kflags = reinterpret_cast<volatile int*>(smem + kMiscOff + 264);   // [kStages]
   float* lse_smem = reinterpret_cast<float*>(smem + kMiscOff + 512);               // [2][128]
+  volatile int* items = reinterpret_cast<volatile int*>(smem + kMiscOff + 1536);   // [2][8]
   auto bar = [&](int which) { return smem_u32(bars + which); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_pairs = (a.Nb + 1) >> 1;
-  // Work order: the heads of one KV head together (their K/V set, 64 MB at 128K, stays in L2 while they run),
-  // inside such a group the longest row-block pairs first, heads fastest.
-  int slot, u;
-  {
-    int id = (int)blockIdx.x, g = 0;
-    while (g + 1 < a.n_groups && id >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
-      id -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
-      ++g;
-    }
-    const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
-    slot = a.order.v[a.group_start.v[g] + id % ng];
-    u = n_pairs - 1 - id / ng;
-  }
-  const int h = a.heads.v[slot];
-  const int g = h / a.group;
-  const int list = a.lists_dev ? a.lists_dev[slot] : a.lists.v[slot];   // decided on the device, or by the host
-  const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
-  TileInfo tile[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    const int i = 2 * u + x;
-    int cnt = 0;
-    if (i < a.Nb && !poisoned) {
-      cnt = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
-      cnt = cnt < 0 ? 0 : (cnt > i + 1 ? i + 1 : cnt);
-    }
-    tile[x].i = i;
-    tile[x].cnt = cnt;
-    tile[x].idx = list >= 0 ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;
-  }
-  const bool any_work = tile[0].cnt + tile[1].cnt > 0;
-  const bool emit = a.importance != nullptr && list < 0;
   const Abort ab{abort_flag, a.status};
   // Optional phase trace (one CTA, one thread per role): {(event << 32) | step, SM clock} pairs.
   const bool tracing = a.trace != nullptr && blockIdx.x == 0;
@@ -228,6 +218,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 
   if (threadIdx.x == 0) {
     mbar_init(bar(BAR_Q_FULL), 1);
+    mbar_init(bar(BAR_Q_EMPTY), 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(BAR_K_FULL + s), 1);
       mbar_init(bar(BAR_K_EMPTY + s), 1);
@@ -237,6 +228,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(BAR_S_FULL + x), 1);
       mbar_init(bar(BAR_O_DONE + x), 1);
+      mbar_init(bar(BAR_ITEM_FULL + x), 1);
+      mbar_init(bar(BAR_ITEM_EMPTY + x), kItemReaders);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -247,64 +240,153 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // The k-th item of this CTA, taken by a whole warp.  False when the wait ran out or another role gave up.
+  auto take_item = [&](int k, Item& it, int where) -> bool {
+    const int sl = k & 1;
+    if (!__all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_FULL + sl), (uint32_t)(k >> 1) & 1u, ab, where))) return false;
+    it.id = items[8 * sl + 0];
+    it.slot = items[8 * sl + 1];
+    it.u = items[8 * sl + 2];
+    it.h = items[8 * sl + 3];
+    it.list = items[8 * sl + 4];
+    it.cntA = items[8 * sl + 5];
+    it.cntB = items[8 * sl + 6];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(BAR_ITEM_EMPTY + sl));
+    return true;
+  };
+
   if (warp >= 8) {
-    if (warp == 9) {
-      // ---------------------------------------------------------- producer
-      if (any_work) {
+    if (warp == 10) {
+      // ---------------------------------------------------------- scheduler
+      // Takes the next position of the work order from the launch's counter, resolves it to (head, pair, list,
+      // counts) and posts it one item ahead of the roles that consume it.  Work order: the heads of one KV head
+      // together (their K/V set, 64 MB at 128K, stays in L2 while they run), inside such a group the longest
+      // row-block pairs first, heads fastest.
+      const int n_items = a.n_heads * n_pairs;
+      const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
+      for (int k = 0;; ++k) {
+        const int sl = k & 1;
+        if (k >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_EMPTY + sl), ((uint32_t)(k >> 1) & 1u) ^ 1u, ab, 40)))
+          break;
+        int id = -1;
         if (lane == 0) {
-          const int n_q = tile[1].i < a.Nb ? 2 : 1;
+          int raw = poisoned ? n_items : atomicAdd(a.work_counter, 1);
+          Item it;
+          it.id = -1; it.slot = 0; it.u = 0; it.h = 0; it.list = -1; it.cntA = 0; it.cntB = 0;
+          if (raw < n_items) {
+            int rest = raw, g = 0;
+            while (g + 1 < a.n_groups && rest >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
+              rest -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
+              ++g;
+            }
+            const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
+            it.id = raw;
+            it.slot = a.order.v[a.group_start.v[g] + rest % ng];
+            it.u = n_pairs - 1 - rest / ng;
+            it.h = a.heads.v[it.slot];
+            it.list = a.lists_dev ? a.lists_dev[it.slot] : a.lists.v[it.slot];   // decided on the device, or by the host
+            if (it.list < 0) it.list = -1;
+            int cnt[2];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const int i = 2 * it.u + x;
+              int c = 0;
+              if (i < a.Nb) {
+                c = it.list >= 0 ? a.counts[(size_t)it.list * a.Nb + i] : i + 1;
+                c = c < 0 ? 0 : (c > i + 1 ? i + 1 : c);
+              }
+              cnt[x] = c;
+            }
+            it.cntA = cnt[0];
+            it.cntB = cnt[1];
+          }
+          items[8 * sl + 0] = it.id;
+          items[8 * sl + 1] = it.slot;
+          items[8 * sl + 2] = it.u;
+          items[8 * sl + 3] = it.h;
+          items[8 * sl + 4] = it.list;
+          items[8 * sl + 5] = it.cntA;
+          items[8 * sl + 6] = it.cntB;
+          mbar_arrive(bar(BAR_ITEM_FULL + sl));
+          id = it.id;
+        }
+        id = __shfl_sync(0xffffffffu, id, 0);
+        if (id < 0) break;
+      }
+    } else if (warp == 9) {
+      // ---------------------------------------------------------- producer
+      int gk = 0;        // merged key-blocks of the finished items (ring position of the next item's first)
+      int issued_k = 0, issued_v = 0;   // K and V loads issued so far
+      int relays = 0;    // relays to the issuing warp so far
+      int qn = 0;        // items with work so far (Q loads)
+      bool ok = true;
+      for (int k = 0; ok; ++k) {
+        Item it;
+        if (!take_item(k, it, 14)) { ok = false; break; }
+        if (it.id < 0) break;
+        const int cntA = it.cntA, cntB = it.cntB;
+        if (cntA + cntB == 0) continue;
+        const int iA = 2 * it.u, iB = iA + 1;
+        const int g = it.h / a.group;
+        // Q of the item before this one has been read by its last QK^T
+        if (qn > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_Q_EMPTY), (uint32_t)(qn - 1) & 1u, ab, 15));
+        if (!ok) break;
+        if (lane == 0) {
+          const int n_q = iB < a.Nb ? 2 : 1;
           mbar_expect_tx(bar(BAR_Q_FULL), n_q * kTile);
           for (int x = 0; x < n_q; ++x)
             for (int b = 0; b < 2; ++b)
-              tma_load_3d(sQ + b * kTile + x * kBox, &tm_q, bar(BAR_Q_FULL), b * 64, tile[x].i * BLK, h);
+              tma_load_3d(sQ + b * kTile + x * kBox, &tm_q, bar(BAR_Q_FULL), b * 64, (iA + x) * BLK, it.h);
         }
+        ++qn;
         // The two ascending lists are merged 32 entries at a time: lane l holds entry base + l.
-        const int cntA = tile[0].cnt, cntB = tile[1].cnt;
-        const int32_t* idxA = tile[0].idx;
-        const int32_t* idxB = tile[1].idx;
-        int pa = 0, pb = 0, n = 0, issued_k = 0, issued_v = 0, relays = 0;
+        const int32_t* idxA = it.list >= 0 ? a.indices + ((size_t)it.list * a.Nb + iA) * a.Nb : nullptr;
+        const int32_t* idxB = it.list >= 0 && iB < a.Nb ? a.indices + ((size_t)it.list * a.Nb + iB) * a.Nb : nullptr;
+        int pa = 0, pb = 0, n = 0;
         int chunkA = 0, chunkB = 0;
         if (idxA) chunkA = lane < cntA ? idxA[lane] : 0;
         if (idxB) chunkB = lane < cntB ? idxB[lane] : 0;
-        bool ok = true;
+        const bool listed = it.list >= 0;
         while ((pa < cntA || pb < cntB) && ok) {
-          const int ja = pa < cntA ? (idxA ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
-          const int jb = pb < cntB ? (idxB ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
+          const int ja = pa < cntA ? (listed ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
+          const int jb = pb < cntB ? (listed ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
           const int j = ja < jb ? ja : jb;
           int f = (ja == j ? F_A : 0) | (jb == j ? F_B : 0);
           if (ja == j) {
             ++pa;
-            if (idxA && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
+            if (listed && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
           }
           if (jb == j) {
             ++pb;
-            if (idxB && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
+            if (listed && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
           }
           if (!(pa < cntA || pb < cntB)) f |= F_LAST;
-          const int st = n % kStages;
-          const uint32_t ph = (uint32_t)(n / kStages) & 1u;
-          if (n >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_K_EMPTY + st), ph ^ 1u, ab, 10));
+          const int gn = gk + n;
+          const int st = gn % kStages;
+          const uint32_t ph = (uint32_t)(gn / kStages) & 1u;
+          if (gn >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_K_EMPTY + st), ph ^ 1u, ab, 10));
           if (!ok) break;
           if (lane == 0) {
             kflags[st] = f;
             mbar_expect_tx(bar(BAR_K_FULL + st), kTile);
             for (int b = 0; b < 2; ++b) tma_load_3d(sK + st * kTile + b * kBox, &tm_k, bar(BAR_K_FULL + st), b * 64, j * BLK, g);
-            trace(0, 20, n);
+            trace(0, 20, gn);
           }
           ++issued_k;
-          if (n >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_V_EMPTY + st), ph ^ 1u, ab, 11));
+          if (gn >= kStages) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_V_EMPTY + st), ph ^ 1u, ab, 11));
           if (!ok) break;
           if (lane == 0) {
             mbar_expect_tx(bar(BAR_V_FULL + st), kTile);
             for (int b = 0; b < 2; ++b) tma_load_3d(sV + st * kTile + b * kBox, &tm_v, bar(BAR_V_FULL + st), b * 64, j * BLK, g);
-            trace(0, 21, n);
+            trace(0, 21, gn);
           }
           ++issued_v;
           ++n;
-          // relay for the issuing warp's iteration n - 2 (key-block n - 2 computed, n - 1 multiplied ahead):
-          // K of key-block n - 1 and V of key-block n - 2 have landed
+          // relay for the issuing warp's iteration n - 2 of this item (key-block n - 2 computed, n - 1 multiplied
+          // ahead): K of key-block n - 1 and V of key-block n - 2 have landed
           if (n >= 2) {
-            const int mk = n - 1, mv = n - 2;
+            const int mk = gk + n - 1, mv = gk + n - 2;
             ok = mbar_wait(bar(BAR_K_FULL + mk % kStages), (uint32_t)(mk / kStages) & 1u, ab, 12);
             if (ok) ok = mbar_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u, ab, 13);
             ok = __all_sync(0xffffffffu, ok);
@@ -313,33 +395,33 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           }
         }
         if (__all_sync(0xffffffffu, ok) && n >= 1) {
-          // the last key-block: only its V is still awaited
-          const int mv = n - 1;
+          // the last key-block of the item: only its V is still awaited
+          const int mv = gk + n - 1;
           ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u, ab, 13));
           bar_arrive(NB_KV + (relays & 3), 64);
           ++relays;
         } else if (n >= 1) {
           bar_arrive(NB_KV + (relays & 3), 64);       // a wait ran out above: release the issuing warp once more
         }
-        if (*abort_flag && lane == 0) {
-          // let the copies already in flight land before the CTA gives its shared memory back
-          const long long t0 = clock64();
-          while (clock64() - t0 < kWaitCycles / 8) {
-            bool done = mbar_try_wait(bar(BAR_Q_FULL), 0);
-            for (int back = 1; back <= kStages; ++back) {   // at most the last kStages loads of a ring are in flight
-              const int mk = issued_k - back, mv = issued_v - back;
-              if (mk >= 0) done = done && mbar_try_wait(bar(BAR_K_FULL + mk % kStages), (uint32_t)(mk / kStages) & 1u);
-              if (mv >= 0) done = done && mbar_try_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u);
-            }
-            if (done) break;
+        gk += n;
+      }
+      if (*abort_flag && lane == 0) {
+        // let the copies already in flight land before the CTA gives its shared memory back
+        const long long t0 = clock64();
+        while (clock64() - t0 < kWaitCycles / 8) {
+          bool done = qn == 0 || mbar_try_wait(bar(BAR_Q_FULL), (uint32_t)(qn - 1) & 1u);
+          for (int back = 1; back <= kStages; ++back) {   // at most the last kStages loads of a ring are in flight
+            const int mk = issued_k - back, mv = issued_v - back;
+            if (mk >= 0) done = done && mbar_try_wait(bar(BAR_K_FULL + mk % kStages), (uint32_t)(mk / kStages) & 1u);
+            if (mv >= 0) done = done && mbar_try_wait(bar(BAR_V_FULL + mv % kStages), (uint32_t)(mv / kStages) & 1u);
           }
+          if (done) break;
         }
       }
     } else if (warp == 8) {
       // ---------------------------------------------------------- MMA issuer
       constexpr uint32_t idesc_qk = instr_desc(128, BLK, 0, 0);
       constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
-      const int cntA = tile[0].cnt, cntB = tile[1].cnt;
       // Descriptors differ from these bases only in the 16-byte-unit address field (low word).
       const uint64_t dq0 = smem_desc(sQ, 16, 1024);
       const uint64_t dk0 = smem_desc(sK, 16, 1024);
@@ -364,293 +446,332 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
                  (accumulate || kk > 0) ? 1u : 0u);
         }
       };
-      bool ok = any_work ? mbar_wait(bar(BAR_Q_FULL), 0, ab, 20) : false;
-      if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, ab, 21);
-      ok = __all_sync(0xffffffffu, ok);
-      int f = 0, n = 0, tA = 0, tB = 0;
-      if (ok) {
+      int gk = 0;            // merged key-blocks so far, over all items (ring position)
+      int relays = 0;        // relays taken from the producer warp so far
+      int tA = 0, tB = 0;    // steps of each tile so far, over all items (parity of its P hand-offs)
+      int qn = 0;            // items with work so far
+      bool ok = true;
+      for (int k = 0; ok; ++k) {
+        Item it;
+        if (!take_item(k, it, 22)) break;
+        if (it.id < 0) break;
+        const int cntA = it.cntA, cntB = it.cntB;
+        if (cntA + cntB == 0) continue;
+        ok = mbar_wait(bar(BAR_Q_FULL), (uint32_t)qn & 1u, ab, 20);
+        if (ok) ok = mbar_wait(bar(BAR_K_FULL + gk % kStages), (uint32_t)(gk / kStages) & 1u, ab, 21);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        ++qn;
         tc_fence_after();
-        f = kflags[0];
+        int f = kflags[gk % kStages];
         if (lane == 0) {
-          trace(1, 1, 0);
-          if (f & F_A) issue_qk(0, 0);
-          if (f & F_B) issue_qk(1, 0);
-          mma_commit(bar(BAR_K_EMPTY + 0));
-          trace(1, 2, 0);
+          trace(1, 1, gk);
+          if (f & F_A) issue_qk(0, gk % kStages);
+          if (f & F_B) issue_qk(1, gk % kStages);
+          mma_commit(bar(BAR_K_EMPTY + gk % kStages));
+          if (f & F_LAST) mma_commit(bar(BAR_Q_EMPTY));
+          trace(1, 2, gk);
         }
         __syncwarp();
-      }
-      // The loop's hand-offs come through named barriers (a poll of an mbarrier costs the issuing warp 150-250
-      // cycles while the tensor pipe streams operands from shared memory; with five polls per key-block the
-      // warp was waiting a quarter of the time with nothing queued): the producer warp relays "K of the next
-      // key-block and V of this one have landed", the softmax warps "P of this tile is stored".  The flags of the
-      // next key-block and the abort flag are read from shared memory ahead of the MMAs whose issue hides the trip.
-      while (ok) {
-        const bool last = (f & F_LAST) != 0;
-        const int st = n % kStages, stn = (n + 1) % kStages;
-        bar_sync(NB_KV + (n & 3), 64);
-        const int fn_early = last ? 0 : kflags[stn];
-        if (f & F_A) {
-          bar_sync(NB_P + 0 + (tA & 1), 160);
-          tc_fence_after();
-          if (lane == 0) {
-            trace(1, 3, n);
-            issue_pv(0, st, 0, tA > 0);
-          }
-          __syncwarp();
-          bar_sync(NB_P + 2 + (tA & 1), 160);
-        }
-        tc_fence_after();
-        const int fn = fn_early;
-        if (lane == 0) {
+        // The loop's hand-offs come through named barriers (a poll of an mbarrier costs the issuing warp 150-250
+        // cycles while the tensor pipe streams operands from shared memory; with five polls per key-block the
+        // warp was waiting a quarter of the time with nothing queued): the producer warp relays "K of the next
+        // key-block and V of this one have landed", the softmax warps "P of this tile is stored".  The flags of the
+        // next key-block and the abort flag are read from shared memory ahead of the MMAs whose issue hides the trip.
+        // The first PV of an item overwrites O of the item before: the softmax warps of the tile have read that O
+        // out of TMEM before they produced the P this PV waits for.
+        int tAl = 0, tBl = 0;  // steps of each tile inside this item
+        for (;;) {
+          const bool last = (f & F_LAST) != 0;
+          const int st = gk % kStages, stn = (gk + 1) % kStages;
+          bar_sync(NB_KV + (relays & 3), 64);
+          ++relays;
+          const int fn_early = last ? 0 : kflags[stn];
           if (f & F_A) {
-            issue_pv(0, st, 1, true);
-            if (tA + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
+            bar_sync(NB_P + 0 + (tA & 1), 160);
+            tc_fence_after();
+            if (lane == 0) {
+              trace(1, 3, gk);
+              issue_pv(0, st, 0, tAl > 0);
+            }
+            __syncwarp();
+            bar_sync(NB_P + 2 + (tA & 1), 160);
           }
-          if (fn & F_A) issue_qk(0, stn);
-          trace(1, 5, n);
-        }
-        __syncwarp();
-        if (f & F_A) ++tA;
-        if (f & F_B) {
-          bar_sync(NB_P + 4 + (tB & 1), 160);
           tc_fence_after();
+          const int fn = fn_early;
           if (lane == 0) {
-            trace(1, 6, n);
-            issue_pv(1, st, 0, tB > 0);
+            if (f & F_A) {
+              issue_pv(0, st, 1, true);
+              if (tAl + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
+            }
+            if (fn & F_A) issue_qk(0, stn);
+            trace(1, 5, gk);
           }
           __syncwarp();
-          bar_sync(NB_P + 6 + (tB & 1), 160);
-        }
-        const int abort_raw = *abort_flag;       // after all syncs of this key-block; looked at after the MMAs below
-        tc_fence_after();
-        if (lane == 0) {
+          if (f & F_A) { ++tA; ++tAl; }
           if (f & F_B) {
-            issue_pv(1, st, 1, true);
-            if (tB + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
+            bar_sync(NB_P + 4 + (tB & 1), 160);
+            tc_fence_after();
+            if (lane == 0) {
+              trace(1, 6, gk);
+              issue_pv(1, st, 0, tBl > 0);
+            }
+            __syncwarp();
+            bar_sync(NB_P + 6 + (tB & 1), 160);
           }
-          mma_commit(bar(BAR_V_EMPTY + st));
-          if (fn & F_B) issue_qk(1, stn);
-          if (!last) mma_commit(bar(BAR_K_EMPTY + stn));
-          trace(1, 4, n);
+          const int abort_raw = *abort_flag;       // after all syncs of this key-block; looked at after the MMAs below
+          tc_fence_after();
+          if (lane == 0) {
+            if (f & F_B) {
+              issue_pv(1, st, 1, true);
+              if (tBl + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
+            }
+            mma_commit(bar(BAR_V_EMPTY + st));
+            if (fn & F_B) issue_qk(1, stn);
+            if (!last) mma_commit(bar(BAR_K_EMPTY + stn));
+            if (fn & F_LAST) mma_commit(bar(BAR_Q_EMPTY));   // Q of this item has been read for the last time
+            trace(1, 4, gk);
+          }
+          __syncwarp();
+          if (f & F_B) { ++tB; ++tBl; }
+          ++gk;
+          if (__any_sync(0xffffffffu, abort_raw != 0)) ok = false;
+          if (last || !ok) break;
+          f = fn;
         }
-        __syncwarp();
-        if (f & F_B) ++tB;
-        if (last || __any_sync(0xffffffffu, abort_raw != 0)) break;
-        f = fn;
-        ++n;
       }
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue of tile x
     const int x = warp >> 2;
     const int row = threadIdx.x & 127;                 // TMEM lane == query row inside the tile
-    const int i = x ? tile[1].i : tile[0].i, cnt = x ? tile[1].cnt : tile[0].cnt;
-    const int32_t* idx = x ? tile[1].idx : tile[0].idx;
-    const int r = i * BLK + row;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t tS = tl + kSCol + x * 128, tO = tl + kOCol + x * 128;
     const float scale = a.scale_log2;
     const int trole = 2 + x;
     const bool tthread = row == 0;
-    float* stats = emit ? a.tile_stats + ((size_t)slot * ((size_t)a.Nb * (a.Nb + 1) / 2) + (size_t)i * (i + 1) / 2) * BLK
-                        : nullptr;
-    float m_ref = -CUDART_INF_F, l = 0.f;
-    bool ok = cnt > 0;
-    int j_next = cnt > 0 ? (idx ? idx[0] : 0) : 0;
-    for (int t = 0; t < cnt && ok; ++t) {
-      const int j = j_next;
-      if (t + 1 < cnt) j_next = idx ? idx[t + 1] : t + 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + x), t & 1, ab, 30 + x));
-      if (!ok) {
-        bar_arrive(NB_P + 4 * x + 0 + (t & 1), 160);   // the issuing warp may be at this step's barriers: do not leave it there
-        bar_arrive(NB_P + 4 * x + 2 + (t & 1), 160);
-        break;
-      }
-      tc_fence_after();
-      if (tthread) trace(trole, 10, t);
-      // The 128 columns are taken as four chunks of 32 (`tcgen05.ld.32x32b.x32`, the next chunk's load in flight).
-      // Chunks 0 and 1 are online-softmax steps of their own: chunk max, (rarely: only when the row max has grown
-      // by more than 2^8) a move of the reference, exponentials, P chunk into columns the sweep has given up.
-      // Then the max of chunks 2 and 3 is taken, and a move they ask for is made, BEFORE the first half of P is
-      // handed over: after that no reference can move in this key-block, so the PV of keys 0..63 may run while
-      // keys 64..127 are exponentiated from the registers they already sit in.
-      const bool diag = j == i;
-      float tile_sum = 0.f;
-      uint32_t sa[32], sb[32];
-      tmem_ld32_async(tS, sa);
-      auto mask_diag = [&](uint32_t* sc, const int c) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e)
-          if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
-      };
-      auto chunk_max = [&](const uint32_t* sc) {
-        float mx0 = max3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
-        float mx1 = max3(__uint_as_float(sc[3]), __uint_as_float(sc[4]), __uint_as_float(sc[5]));
-        float mx2 = max3(__uint_as_float(sc[6]), __uint_as_float(sc[7]), __uint_as_float(sc[8]));
-        float mx3 = max3(__uint_as_float(sc[9]), __uint_as_float(sc[10]), __uint_as_float(sc[11]));
-#pragma unroll
-        for (int e = 12; e < 28; e += 8) {
-          mx0 = max3(mx0, __uint_as_float(sc[e + 0]), __uint_as_float(sc[e + 1]));
-          mx1 = max3(mx1, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]));
-          mx2 = max3(mx2, __uint_as_float(sc[e + 4]), __uint_as_float(sc[e + 5]));
-          mx3 = max3(mx3, __uint_as_float(sc[e + 6]), __uint_as_float(sc[e + 7]));
+    // per-CTA statistics region: [tile][step of the item][row]
+    float* const stats = a.tile_stats ? a.tile_stats + ((size_t)blockIdx.x * 2 + x) * (size_t)a.Nb * BLK : nullptr;
+    int ts = 0;          // steps of this tile so far, over all items (parity of S_FULL and of the P hand-offs)
+    int on = 0;          // items in which this tile had work so far (parity of O_DONE)
+    bool fail = false;   // a wait of this thread ran out
+    for (int k = 0;; ++k) {
+      Item it;
+      it.id = -1;
+      const bool got = !fail && take_item(k, it, 34 + x);
+      // The four warps of the tile go on together or stop together (a warp whose wait ran out must not leave the
+      // others at the barriers of the epilogue).  This barrier also separates the reads of the statistics region
+      // by the epilogue of the item before from the writes of this item.
+      if (!bar_and(1 + x, 128, got)) break;
+      if (it.id < 0) break;
+      const int i = 2 * it.u + x, cnt = x ? it.cntB : it.cntA;
+      const int h = it.h, slot = it.slot;
+      const int32_t* idx = it.list >= 0 && i < a.Nb ? a.indices + ((size_t)it.list * a.Nb + i) * a.Nb : nullptr;
+      const bool emit = a.importance != nullptr && it.list < 0;
+      const int r = i * BLK + row;
+      float m_ref = -CUDART_INF_F, l = 0.f;
+      bool ok = cnt > 0;
+      int j_next = cnt > 0 ? (idx ? idx[0] : 0) : 0;
+      for (int t = 0; t < cnt && ok; ++t, ++ts) {
+        const int j = j_next;
+        if (t + 1 < cnt) j_next = idx ? idx[t + 1] : t + 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + x), (uint32_t)ts & 1u, ab, 30 + x));
+        if (!ok) {
+          fail = true;
+          bar_arrive(NB_P + 4 * x + 0 + (ts & 1), 160);   // the issuing warp may be at this step's barriers: do not leave it there
+          bar_arrive(NB_P + 4 * x + 2 + (ts & 1), 160);
+          break;
         }
-        mx0 = max3(mx0, __uint_as_float(sc[28]), __uint_as_float(sc[29]));
-        mx1 = max3(mx1, __uint_as_float(sc[30]), __uint_as_float(sc[31]));
-        return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      };
-      // mx: scaled max of the columns about to be exponentiated; stored: P chunks of this key-block already in TMEM
-      auto move_reference = [&](const float mx, const int stored) {
-        // the reference max only moves when the row max has grown by more than 2^8 (rare after the first chunk of
-        // the first key-block; a fully masked chunk has mx = -inf and leaves it alone)
-        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
-          const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
-          const float alpha = ex2_approx(m_ref - m_new);
-          if (t > 0) {
-            // O of the previous steps is relative to the old reference: bring it to the new one.
-            // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
-#pragma unroll 1
-            for (int oc = 0; oc < D / 32; ++oc) {
-              uint32_t o[32];
-              tmem_ld32(tO + oc * 32, o);
+        tc_fence_after();
+        if (tthread) trace(trole, 10, t);
+        // The 128 columns are taken as four chunks of 32 (`tcgen05.ld.32x32b.x32`, the next chunk's load in flight).
+        // Chunks 0 and 1 are online-softmax steps of their own: chunk max, (rarely: only when the row max has grown
+        // by more than 2^8) a move of the reference, exponentials, P chunk into columns the sweep has given up.
+        // Then the max of chunks 2 and 3 is taken, and a move they ask for is made, BEFORE the first half of P is
+        // handed over: after that no reference can move in this key-block, so the PV of keys 0..63 may run while
+        // keys 64..127 are exponentiated from the registers they already sit in.
+        const bool diag = j == i;
+        float tile_sum = 0.f;
+        uint32_t sa[32], sb[32];
+        tmem_ld32_async(tS, sa);
+        auto mask_diag = [&](uint32_t* sc, const int c) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st32(tO + oc * 32, o);
+          for (int e = 0; e < 32; ++e)
+            if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
+        };
+        auto chunk_max = [&](const uint32_t* sc) {
+          float mx0 = max3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
+          float mx1 = max3(__uint_as_float(sc[3]), __uint_as_float(sc[4]), __uint_as_float(sc[5]));
+          float mx2 = max3(__uint_as_float(sc[6]), __uint_as_float(sc[7]), __uint_as_float(sc[8]));
+          float mx3 = max3(__uint_as_float(sc[9]), __uint_as_float(sc[10]), __uint_as_float(sc[11]));
+#pragma unroll
+          for (int e = 12; e < 28; e += 8) {
+            mx0 = max3(mx0, __uint_as_float(sc[e + 0]), __uint_as_float(sc[e + 1]));
+            mx1 = max3(mx1, __uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3]));
+            mx2 = max3(mx2, __uint_as_float(sc[e + 4]), __uint_as_float(sc[e + 5]));
+            mx3 = max3(mx3, __uint_as_float(sc[e + 6]), __uint_as_float(sc[e + 7]));
+          }
+          mx0 = max3(mx0, __uint_as_float(sc[28]), __uint_as_float(sc[29]));
+          mx1 = max3(mx1, __uint_as_float(sc[30]), __uint_as_float(sc[31]));
+          return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        };
+        // mx: scaled max of the columns about to be exponentiated; stored: P chunks of this key-block already in TMEM
+        auto move_reference = [&](const float mx, const int stored) {
+          // the reference max only moves when the row max has grown by more than 2^8 (rare after the first chunk of
+          // the first key-block; a fully masked chunk has mx = -inf and leaves it alone)
+          if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+            const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
+            const float alpha = ex2_approx(m_ref - m_new);
+            if (t > 0) {
+              // O of the previous steps is relative to the old reference: bring it to the new one.
+              // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
+#pragma unroll 1
+              for (int oc = 0; oc < D / 32; ++oc) {
+                uint32_t o[32];
+                tmem_ld32(tO + oc * 32, o);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                tmem_st32(tO + oc * 32, o);
+              }
+            }
+            // the P chunks of this key-block that are already stored (none of them handed over yet)
+#pragma unroll 1
+            for (int pc = 0; pc < stored; ++pc) {
+              uint32_t pp[16];
+              tmem_ld16(tS + pc * 16, pp);
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
+              tmem_st16(tS + pc * 16, pp);
+            }
+            l *= alpha;
+            tile_sum *= alpha;
+            m_ref = m_new;
+          }
+        };
+        auto chunk_exps = [&](const uint32_t* sc, const int c) {   // exponentials, sums, P chunk c (columns 32c .. 32c+31)
+          const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_ref, -m_ref);
+          float2 sum01 = make_float2(0.f, 0.f), sum23 = make_float2(0.f, 0.f);
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sc[e]), __uint_as_float(sc[e + 1])), sc2, nm2);
+            float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3])), sc2, nm2);
+            x01.x = ex2_approx(x01.x);
+            x01.y = ex2_approx(x01.y);
+            x23.x = ex2_approx(x23.x);
+            x23.y = ex2_approx(x23.y);
+            sum01 = __fadd2_rn(sum01, x01);
+            sum23 = __fadd2_rn(sum23, x23);
+            pk[e / 2] = cvt_bf16x2(x01.x, x01.y);
+            pk[e / 2 + 1] = cvt_bf16x2(x23.x, x23.y);
+          }
+          tile_sum += (sum01.x + sum01.y) + (sum23.x + sum23.y);
+          tmem_st16(tS + c * 16, pk);
+        };
+        tmem_ld_wait();
+        reg_fence32(sa);
+        tmem_ld32_async(tS + 32, sb);
+        if (diag) mask_diag(sa, 0);
+        move_reference(chunk_max(sa) * scale, 0);
+        chunk_exps(sa, 0);
+        tmem_ld_wait();
+        reg_fence32(sb);
+        tmem_ld32_async(tS + 64, sa);
+        if (diag) mask_diag(sb, 1);
+        move_reference(chunk_max(sb) * scale, 1);
+        chunk_exps(sb, 1);
+        tmem_ld_wait();
+        reg_fence32(sa);
+        tmem_ld32_async(tS + 96, sb);
+        if (diag) mask_diag(sa, 2);
+        float mx23 = chunk_max(sa);
+        tmem_ld_wait();
+        reg_fence32(sb);
+        if (diag) mask_diag(sb, 3);
+        mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
+        move_reference(mx23, 2);
+        tmem_wait_st();
+        tc_fence_before();
+        bar_arrive(NB_P + 4 * x + 0 + (ts & 1), 160);
+        if (tthread) trace(trole, 13, t);
+        chunk_exps(sa, 2);
+        chunk_exps(sb, 3);
+        tmem_wait_st();
+        tc_fence_before();
+        bar_arrive(NB_P + 4 * x + 2 + (ts & 1), 160);
+        if (tthread) trace(trole, 15, t);
+        // off the critical path: running sum and the tile statistic
+        l += tile_sum;
+        if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(tile_sum);
+      }
+      if (ok) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_O_DONE + x), (uint32_t)on & 1u, ab, 32 + x));
+        if (!ok) fail = true;
+      }
+      if (cnt > 0) ++on;
+      float lse2 = 0.f;
+      if (ok) {
+        tc_fence_after();
+        const float inv_l = 1.f / l;
+        __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + c * 32, o);
+          uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            uint4 w;
+            w.x = cvt_bf16x2(__uint_as_float(o[8 * e + 0]) * inv_l, __uint_as_float(o[8 * e + 1]) * inv_l);
+            w.y = cvt_bf16x2(__uint_as_float(o[8 * e + 2]) * inv_l, __uint_as_float(o[8 * e + 3]) * inv_l);
+            w.z = cvt_bf16x2(__uint_as_float(o[8 * e + 4]) * inv_l, __uint_as_float(o[8 * e + 5]) * inv_l);
+            w.w = cvt_bf16x2(__uint_as_float(o[8 * e + 6]) * inv_l, __uint_as_float(o[8 * e + 7]) * inv_l);
+            dst[e] = w;
+          }
+        }
+        // O has left TMEM: ordered before the P hand-off of the next item, after which its first PV overwrites O
+        tc_fence_before();
+        lse2 = m_ref + log2f(l);
+        if (a.lse) a.lse[(size_t)slot * a.N + r] = lse2 * 0.6931471805599453f;
+      }
+      if (emit) {
+        float* lse_x = lse_smem + x * 128;
+        lse_x[row] = lse2;
+        // the four softmax warps of this tile: statistics and lse visible to one another, and one
+        // common decision (a thread whose wait ran out must not leave the others at a barrier)
+        const bool all_ok = bar_and(1 + x, 128, ok);
+        if (all_ok) {
+          float* imp_row = a.importance + ((size_t)slot * a.Nb + i) * a.Nb;
+          const float4 lse4 = *reinterpret_cast<const float4*>(lse_x + lane * 4);
+          const int wq = warp & 3;
+          // each warp takes tiles wq, wq + 4, ...; eight tiles in flight; lane l sums rows 4l..4l+3
+          for (int t0 = wq; t0 < cnt; t0 += 32) {
+            float4 v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int t = t0 + 4 * e;
+              v[e] = t < cnt ? *reinterpret_cast<const float4*>(stats + (size_t)t * BLK + lane * 4)
+                             : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              float acc = (ex2_approx(v[e].x - lse4.x) + ex2_approx(v[e].y - lse4.y)) +
+                          (ex2_approx(v[e].z - lse4.z) + ex2_approx(v[e].w - lse4.w));
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+              const int t = t0 + 4 * e;
+              if (lane == 0 && t < cnt) imp_row[t] = acc * (1.f / BLK);
             }
           }
-          // the P chunks of this key-block that are already stored (none of them handed over yet)
-#pragma unroll 1
-          for (int pc = 0; pc < stored; ++pc) {
-            uint32_t pp[16];
-            tmem_ld16(tS + pc * 16, pp);
-#pragma unroll
-            for (int e = 0; e < 16; ++e)
-              pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
-            tmem_st16(tS + pc * 16, pp);
-          }
-          l *= alpha;
-          tile_sum *= alpha;
-          m_ref = m_new;
-        }
-      };
-      auto chunk_exps = [&](const uint32_t* sc, const int c) {   // exponentials, sums, P chunk c (columns 32c .. 32c+31)
-        const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(-m_ref, -m_ref);
-        float2 sum01 = make_float2(0.f, 0.f), sum23 = make_float2(0.f, 0.f);
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sc[e]), __uint_as_float(sc[e + 1])), sc2, nm2);
-          float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sc[e + 2]), __uint_as_float(sc[e + 3])), sc2, nm2);
-          x01.x = ex2_approx(x01.x);
-          x01.y = ex2_approx(x01.y);
-          x23.x = ex2_approx(x23.x);
-          x23.y = ex2_approx(x23.y);
-          sum01 = __fadd2_rn(sum01, x01);
-          sum23 = __fadd2_rn(sum23, x23);
-          pk[e / 2] = cvt_bf16x2(x01.x, x01.y);
-          pk[e / 2 + 1] = cvt_bf16x2(x23.x, x23.y);
-        }
-        tile_sum += (sum01.x + sum01.y) + (sum23.x + sum23.y);
-        tmem_st16(tS + c * 16, pk);
-      };
-      tmem_ld_wait();
-      reg_fence32(sa);
-      tmem_ld32_async(tS + 32, sb);
-      if (diag) mask_diag(sa, 0);
-      move_reference(chunk_max(sa) * scale, 0);
-      chunk_exps(sa, 0);
-      tmem_ld_wait();
-      reg_fence32(sb);
-      tmem_ld32_async(tS + 64, sa);
-      if (diag) mask_diag(sb, 1);
-      move_reference(chunk_max(sb) * scale, 1);
-      chunk_exps(sb, 1);
-      tmem_ld_wait();
-      reg_fence32(sa);
-      tmem_ld32_async(tS + 96, sb);
-      if (diag) mask_diag(sa, 2);
-      float mx23 = chunk_max(sa);
-      tmem_ld_wait();
-      reg_fence32(sb);
-      if (diag) mask_diag(sb, 3);
-      mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
-      move_reference(mx23, 2);
-      tmem_wait_st();
-      tc_fence_before();
-      bar_arrive(NB_P + 4 * x + 0 + (t & 1), 160);
-      if (tthread) trace(trole, 13, t);
-      chunk_exps(sa, 2);
-      chunk_exps(sb, 3);
-      tmem_wait_st();
-      tc_fence_before();
-      bar_arrive(NB_P + 4 * x + 2 + (t & 1), 160);
-      if (tthread) trace(trole, 15, t);
-      // off the critical path: running sum and the tile statistic
-      l += tile_sum;
-      if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(tile_sum);
-    }
-    if (ok) ok = mbar_wait(bar(BAR_O_DONE + x), 0, ab, 32 + x);
-    float lse2 = 0.f;
-    if (ok) {
-      tc_fence_after();
-      const float inv_l = 1.f / l;
-      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tO + c * 32, o);
-        uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          uint4 w;
-          w.x = cvt_bf16x2(__uint_as_float(o[8 * e + 0]) * inv_l, __uint_as_float(o[8 * e + 1]) * inv_l);
-          w.y = cvt_bf16x2(__uint_as_float(o[8 * e + 2]) * inv_l, __uint_as_float(o[8 * e + 3]) * inv_l);
-          w.z = cvt_bf16x2(__uint_as_float(o[8 * e + 4]) * inv_l, __uint_as_float(o[8 * e + 5]) * inv_l);
-          w.w = cvt_bf16x2(__uint_as_float(o[8 * e + 6]) * inv_l, __uint_as_float(o[8 * e + 7]) * inv_l);
-          dst[e] = w;
+          for (int jz = i + 1 + row; jz < a.Nb; jz += 128) imp_row[jz] = 0.f;
         }
       }
-      lse2 = m_ref + log2f(l);
-      if (a.lse) a.lse[(size_t)slot * a.N + r] = lse2 * 0.6931471805599453f;
-    }
-    if (emit) {
-      float* lse_x = lse_smem + x * 128;
-      lse_x[row] = lse2;
-      // the four softmax warps of this tile: statistics and lse visible to one another, and one
-      // common decision (a thread whose wait ran out must not leave the others at a barrier)
-      const bool all_ok = bar_and(1 + x, 128, ok);
-      if (all_ok) {
-        float* imp_row = a.importance + ((size_t)slot * a.Nb + i) * a.Nb;
-        const float4 lse4 = *reinterpret_cast<const float4*>(lse_x + lane * 4);
-        const int wq = warp & 3;
-        // each warp takes tiles wq, wq + 4, ...; eight tiles in flight; lane l sums rows 4l..4l+3
-        for (int t0 = wq; t0 < cnt; t0 += 32) {
-          float4 v[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const int t = t0 + 4 * e;
-            v[e] = t < cnt ? *reinterpret_cast<const float4*>(stats + (size_t)t * BLK + lane * 4)
-                           : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
-          }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            float acc = (ex2_approx(v[e].x - lse4.x) + ex2_approx(v[e].y - lse4.y)) +
-                        (ex2_approx(v[e].z - lse4.z) + ex2_approx(v[e].w - lse4.w));
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            const int t = t0 + 4 * e;
-            if (lane == 0 && t < cnt) imp_row[t] = acc * (1.f / BLK);
-          }
-        }
-        for (int jz = i + 1 + row; jz < a.Nb; jz += 128) imp_row[jz] = 0.f;
+      if (!ok && !fail && cnt == 0 && i < a.Nb) {
+        // an empty list is outside the contract; leave defined output (zeros) rather than garbage
+        __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
+        for (int e = 0; e < D / 8; ++e) reinterpret_cast<uint4*>(orow)[e] = make_uint4(0, 0, 0, 0);
       }
-    }
-    if (ok) {
-    } else if (cnt == 0 && i < a.Nb && !poisoned) {
-      // an empty list is outside the contract; leave defined output (zeros) rather than garbage
-      __nv_bfloat16* orow = a.o + (size_t)h * a.o_sh + (size_t)r * a.o_sn;
-      for (int e = 0; e < D / 8; ++e) reinterpret_cast<uint4*>(orow)[e] = make_uint4(0, 0, 0, 0);
     }
   }
 
@@ -666,17 +787,31 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 
 bool attn_pair_supported(const AttnArgs& a) { return a.d == D && a.B == BLK; }
 
+namespace {
+int sm_count() {
+  int n_sm = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  return n_sm > 0 ? n_sm : 148;
+}
+}  // namespace
+
+int attn_pair_ctas(int n_heads, int Nb) {
+  const long items = (long)n_heads * ((Nb + 1) / 2);
+  const int n_sm = sm_count();
+  return (int)(items < n_sm ? items : n_sm);
+}
+
+size_t attn_pair_stats_bytes(int n_heads, int Nb) {
+  return (size_t)attn_pair_ctas(n_heads, Nb) * 2 * (size_t)Nb * BLK * sizeof(float);
+}
+
 cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
-  if (!attn_pair_supported(a_in)) return cudaErrorInvalidValue;
+  if (!attn_pair_supported(a_in) || !a_in.work_counter) return cudaErrorInvalidValue;
   AttnArgs a = a_in;
-  // Work order.  Many CTAs (forty waves or more): the slots sorted by KV head (stable), one group per KV head,
+  // Work order.  Many items (forty per SM or more): the slots sorted by KV head (stable), one group per KV head,
   // so that a K/V set stays in L2 while its heads run.  Fewer: one group, i.e. the longest pairs of all heads
-  // first, because with a few waves the balance of the last wave matters more than L2.
-  int n_sm = 148;
-  {
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-  }
+  // first, because then the balance at the end matters more than L2.
+  const int n_sm = sm_count();
   const bool by_kv_head = (long)a.n_heads * ((a.Nb + 1) / 2) >= 40L * n_sm;
   int n = 0;
   a.n_groups = 0;
@@ -691,6 +826,7 @@ cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
     for (int t = 0; t < a.n_heads; ++t) a.order.v[n++] = t;
     a.group_start.v[a.n_groups++] = 0;
   }
+  static_assert(sizeof(a.group_start.v) / sizeof(a.group_start.v[0]) == kMaxHeads + 1, "room for the end of the last group");
   a.group_start.v[a.n_groups] = n;
   CUtensorMap tq, tk, tv;
   if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
@@ -699,7 +835,10 @@ cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
   if (e != cudaSuccess) return e;
-  attn_pair_kernel<<<a.n_heads * ((a.Nb + 1) / 2), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
+  // Persistent CTAs, one per SM, take the items of the work order from a counter that starts at zero.
+  e = cudaMemsetAsync(a.work_counter, 0, sizeof(int), s);
+  if (e != cudaSuccess) return e;
+  attn_pair_kernel<<<attn_pair_ctas(a.n_heads, a.Nb), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
   return cudaGetLastError();
 }
 

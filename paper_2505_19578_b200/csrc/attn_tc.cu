@@ -348,12 +348,13 @@ cudaError_t launch(const AttnArgs& a, cudaStream_t s) {
 //
 // Scratch for callers that cannot allocate: the per-tile softmax statistics of a
 // dense pivot launch live in this file-scope array instead of a cudaMalloc'ed
-// workspace.  Every device that loads the library carries the array until the
-// process exits.  In host code `g_fixed_scratch` is only a handle for the runtime,
-// not a device address: the address a kernel may use comes from
-// cudaGetSymbolAddress, asked once per device with that device current.
+// workspace, and so do the status word and the work counter of the launch.
+// Every device that loads the library carries the array until the process exits.
+// In host code `g_fixed_scratch` is only a handle for the runtime, not a device
+// address: the address a kernel may use comes from cudaGetSymbolAddress, asked
+// once per device with that device current.
 static __device__ __align__(256) unsigned char g_fixed_scratch[kFixedScratchBytes];
-static __device__ __align__(256) int g_fixed_status[2];
+static __device__ __align__(256) int g_fixed_status[4];   // {code, where, work counter, unused}
 
 namespace {
 constexpr int kMaxDevices = 64;
@@ -361,31 +362,62 @@ void* g_fixed_scratch_addr[kMaxDevices];
 void* g_fixed_status_addr[kMaxDevices];
 bool g_fixed_ready[kMaxDevices];
 std::mutex g_fixed_mutex;
-}  // namespace
 
-cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s) {
+// first call on this device (the caller made it current): resolve both symbols
+cudaError_t fixed_setup(int device) {
   if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
   std::lock_guard<std::mutex> lock(g_fixed_mutex);
-  if (!g_fixed_ready[device]) {
-    // first call on this device (the caller made it current): resolve both symbols
-    void* scratch = nullptr;
-    void* status = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&scratch, g_fixed_scratch);
-    if (e != cudaSuccess) return e;
-    e = cudaGetSymbolAddress(&status, g_fixed_status);
-    if (e != cudaSuccess) return e;
-    g_fixed_scratch_addr[device] = scratch;
-    g_fixed_status_addr[device] = status;
-    g_fixed_ready[device] = true;
-  }
+  if (g_fixed_ready[device]) return cudaSuccess;
+  void* scratch = nullptr;
+  void* status = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&scratch, g_fixed_scratch);
+  if (e != cudaSuccess) return e;
+  e = cudaGetSymbolAddress(&status, g_fixed_status);
+  if (e != cudaSuccess) return e;
+  g_fixed_scratch_addr[device] = scratch;
+  g_fixed_status_addr[device] = status;
+  g_fixed_ready[device] = true;
+  return cudaSuccess;
+}
+}  // namespace
+
+// Bytes of the fixed array a launch needs (with the launch's device current).
+size_t fixed_scratch_need(const AttnArgs& a) {
+  if (!a.importance) return 0;
+  return attn_pair_supported(a) ? attn_pair_stats_bytes(a.n_heads, a.Nb)
+                                : (size_t)a.n_heads * tile_stats_bytes_per_head(a.Nb, a.B);
+}
+
+cudaError_t launch_attn_fixed_scratch(AttnArgs a, int device, cudaStream_t s) {
+  cudaError_t e = fixed_setup(device);
+  if (e != cudaSuccess) return e;
+  if (fixed_scratch_need(a) > kFixedScratchBytes) return cudaErrorInvalidValue;
   a.tile_stats = static_cast<float*>(g_fixed_scratch_addr[device]);
   a.status = static_cast<int*>(g_fixed_status_addr[device]);
-  // the status word keeps the previous call's value and the kernel refuses to work
-  // when it is non-zero: it has to start at zero.  The statistics need no clearing:
-  // every entry that is read has been written by the same launch.
-  cudaError_t e = cudaMemsetAsync(a.status, 0, 2 * sizeof(int), s);
+  a.work_counter = a.status + 2;
+  // the status word keeps the previous call's value and the kernels refuse to work
+  // when it is non-zero: it has to start at zero (the paired launch clears its work
+  // counter itself).  The statistics need no clearing: every entry that is read has
+  // been written by the same launch.
+  e = cudaMemsetAsync(a.status, 0, 2 * sizeof(int), s);
   if (e != cudaSuccess) return e;
-  return launch_attn_tc(a, s);
+  return attn_pair_supported(a) ? launch_attn_pair(a, s) : launch_attn_tc(a, s);
+}
+
+// Reads the fixed status word of `device` back (and clears it when it is set).  The caller has synchronised.
+cudaError_t fixed_status_read(int device, int* code, int* where) {
+  cudaError_t e = fixed_setup(device);
+  if (e != cudaSuccess) return e;
+  int host[2] = {0, 0};
+  e = cudaMemcpy(host, g_fixed_status_addr[device], sizeof(host), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return e;
+  if (host[0] != 0) {
+    e = cudaMemset(g_fixed_status_addr[device], 0, sizeof(host));
+    if (e != cudaSuccess) return e;
+  }
+  if (code) *code = host[0];
+  if (where) *where = host[1];
+  return cudaSuccess;
 }
 
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s) {

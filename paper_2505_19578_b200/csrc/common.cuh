@@ -6,7 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "shareprefill.h"
+#include "shareprefill_internal.h"
 
 namespace sp {
 
@@ -15,6 +15,9 @@ constexpr int kMaxNb = 1024;     // key-blocks per row (mask kernel sorts one ro
 
 struct HeadTable {
   int32_t v[kMaxHeads];
+};
+struct GroupTable {          // group boundaries: one entry more than there can be groups
+  int32_t v[kMaxHeads + 1];
 };
 
 // Everything an attention launch needs.  Strides are in elements.
@@ -31,14 +34,16 @@ struct AttnArgs {
   HeadTable lists;         // list index per slot, -1 = dense (all causal tiles)
   const int32_t* lists_dev;  // if not null: list index per slot read from device memory instead
   HeadTable order;         // paired kernel: slots sorted by KV head (position -> slot)
-  HeadTable group_start;   // paired kernel: first sorted position of each KV-head group, then n_heads
+  GroupTable group_start;  // paired kernel: first sorted position of each KV-head group, then n_heads
   int n_groups;
   const int32_t* counts;   // [n_lists, Nb]       (may be null when every slot is dense)
   const int32_t* indices;  // [n_lists, Nb, Nb]
   float* importance;       // [n_heads, Nb, Nb] or null
   float* lse;              // [n_heads, N] or null
-  float* tile_stats;       // scratch: per (slot, row-block) B floats per causal tile (tensor-core path)
+  float* tile_stats;       // scratch of the importance map: one-row-block kernel, per (slot, row-block) B floats per causal
+                           // tile; paired kernel, per CTA 2 * Nb * B floats (attn_pair_stats_bytes)
   int* status;             // device int[2]: {code, where}
+  int* work_counter;       // paired kernel: device int, the launch's position in its work order (cleared by the launcher)
   long long* trace;        // optional phase trace of CTA (0,0): 5 roles x trace_cap x {tag, clock}
   int trace_cap;
   float scale_log2;        // log2(e) / sqrt(d)
@@ -91,8 +96,15 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t s);   // tcgen05 / TM
 // tcgen05 / TMEM / TMA, two adjacent row-blocks per CTA sharing their K/V tiles (head_dim 128, block 128)
 bool attn_pair_supported(const AttnArgs& a);
 cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s);
-// same kernel, statistics and status word in the library's fixed device arrays
-cudaError_t launch_attn_tc_fixed_scratch(AttnArgs a, int device, cudaStream_t s);
+// CTAs a paired launch over n_heads heads runs (one per SM of the current device at most), and the bytes of
+// tile statistics it needs when it emits importance: one region of 2 * Nb * 128 floats per CTA
+int attn_pair_ctas(int n_heads, int Nb);
+size_t attn_pair_stats_bytes(int n_heads, int Nb);
+// dense attention with importance, statistics, status word and work counter in the library's fixed device arrays
+// (the paired kernel at head_dim 128 / block 128, the one-row-block kernel otherwise)
+size_t fixed_scratch_need(const AttnArgs& a);
+cudaError_t launch_attn_fixed_scratch(AttnArgs a, int device, cudaStream_t s);
+cudaError_t fixed_status_read(int device, int* code, int* where);
 constexpr size_t kFixedScratchBytes = 64ull << 20;
 cudaError_t launch_block_mask(const MaskArgs& a, cudaStream_t s);
 cudaError_t launch_fill_causal_mask(uint8_t* mask, int nb, cudaStream_t s);

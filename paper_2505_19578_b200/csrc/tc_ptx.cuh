@@ -203,7 +203,7 @@ inline EncodeTiledFn encode_fn() {
 inline bool make_map(CUtensorMap* m, const void* base, int64_t sh, int64_t sn, int H, int N, int d, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  if (H == 1 || sh == 0) sh = (int64_t)N * sn;
+  if (H == 1) sh = (int64_t)N * sn;   // a single head: its stride is never used, but the encoder wants a valid one
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H};
   cuuint64_t strides[2] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};

@@ -43,8 +43,13 @@ def test_host_only_calls(lib):
     assert "timed out" in binding.error_string(binding.SP_ERR_TIMEOUT)
     b = binding.workspace_bytes(131072, 32, 8, 128, 128, 4)
     nb = 1024
-    # importance + mask + counts + lists + per-tile statistics
-    assert b >= 4 * nb * nb * (4 + 1 + 4) + 4 * nb * (nb + 1) // 2 * 128 * 4
+    # importance + mask + counts + lists, and per-tile statistics: one region of 2 * nb * 128 floats per
+    # persistent CTA (at most one per SM) instead of one float per row of every causal tile of every pivot
+    assert b >= 4 * nb * nb * (4 + 1 + 4) + 2 * nb * 128 * 4
+    assert b < 256 << 20
+    # the one-row-block kernel (other shapes) keeps the per-tile layout
+    b64 = binding.workspace_bytes(8192, 8, 8, 64, 64, 2)
+    assert b64 >= 2 * 128 * 129 // 2 * 64 * 4
     out = ctypes.c_size_t()
     assert lib.sp_workspace_bytes(1000, 32, 8, 128, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED
     assert lib.sp_workspace_bytes(4096, 32, 8, 96, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED

@@ -324,6 +324,8 @@ def test_invalid_arguments_are_rejected(binding):
     assert code(lambda: ctx.sp_dense_pivot_attn(q96, k96, k96, [0], 128, torch.zeros_like(q96))) == binding.SP_ERR_UNSUPPORTED
     assert code(lambda: ctx.sp_dense_pivot_attn(q, k, k[:, :128], [0], 128, out)) == binding.SP_ERR_INVALID_ARG
     assert code(lambda: ctx.sp_prefill_attn(q, k, k, [0, 0, 1, 1], [0, 0], 0.9, 128, out)) == binding.SP_ERR_INVALID_ARG  # dup
+    k_bcast = k[:1].expand(2, 256, 128)                      # one KV head broadcast over two: head stride 0
+    assert code(lambda: ctx.sp_dense_pivot_attn(q, k_bcast, k_bcast, [0], 128, out)) == binding.SP_ERR_INVALID_ARG
     assert code(lambda: ctx.sp_prefill_attn(q, k, k, [0, 0, 1, 1], [0], 0.0, 128, out)) == binding.SP_ERR_INVALID_ARG
     imp = torch.zeros(1, 8, 8, device="cuda")
     cnt = torch.zeros(1, 8, dtype=torch.int32, device="cuda")
