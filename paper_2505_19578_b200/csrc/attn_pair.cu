@@ -18,16 +18,22 @@
 // key-block only one of them selected is computed for that tile alone.  (Dense:
 // the union is 0..2u+1, the last key-block is B's diagonal tile only.)
 //
-// Warp roles (352 threads):
+// Warp roles (320 threads):
 //   warps 0-3   softmax of tile A: thread t owns query row t = TMEM lane t
 //   warps 4-7   softmax of tile B
 //   warp  8     MMA issuer, owner of the TMEM allocation (all 512 columns:
 //               S_A, S_B, O_A, O_B, 128 fp32 columns each)
-//   warp  9     producer: merges the two lists, TMA loads of Q (once per item)
+//   warp  9     producer: takes the next item from the counter, resolves it to
+//               (head, pair, list, counts) and posts it in a two-slot ring of
+//               shared memory that the other nine warps read (it runs ahead of
+//               them by the depth of the K/V rings, so they find the item
+//               waiting); merges the two lists; TMA loads of Q (once per item)
 //               and of the K and V tiles into two-stage rings (128-byte swizzle)
-//   warp 10     scheduler: takes the next item from the counter, resolves it to
-//               (head, pair, list, counts) and posts it, one item ahead, in a
-//               two-slot ring of shared memory that the other ten warps read
+//
+// The kernel is sensitive to the size of its hot loops (an eleventh warp for the
+// scheduling, bounded waits inlined at every site and the phase trace compiled
+// into the loops cost 3 %, 3 % and 2 % of the layer): rare paths are kept out
+// of line.
 //
 // Rings, barrier phases and named-barrier ids run on across items (every role
 // counts key-blocks, tile steps and items for itself).
@@ -77,8 +83,8 @@ using namespace tc;
 
 constexpr int D = 128;      // head_dim
 constexpr int BLK = 128;    // block
-constexpr int kThreadsPair = 352;   // eight softmax warps, the issuing, the producer and the scheduler warp
-constexpr int kItemReaders = 10;     // warps that take every work item: all but the scheduler
+constexpr int kThreadsPair = 320;   // eight softmax warps, the issuing warp, the producer warp
+constexpr int kItemReaders = 9;       // warps that take every posted item: all but the producer, which posts it
 constexpr int kStages = 2;  // K ring and V ring depth
 
 // shared-memory plan (bytes)
@@ -187,6 +193,48 @@ struct Item {
   int cntB;    // key-blocks tile B visits
 };
 
+// Rare path of the softmax, kept out of the hot loop: the row's reference max has moved, so O of the earlier
+// steps (when there are any) and the P chunks of this key-block that are already stored are brought to the new
+// reference.  alpha = 2^(old reference - new reference), 1 for a row whose reference stays.  Called by whole warps.
+static __device__ __noinline__ void rescale_tmem(uint32_t tO, uint32_t tS, float alpha, int stored, bool with_o) {
+  if (with_o) {
+#pragma unroll 1
+    for (int oc = 0; oc < D / 32; ++oc) {
+      uint32_t o[32];
+      tmem_ld32(tO + oc * 32, o);
+#pragma unroll
+      for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+      tmem_st32(tO + oc * 32, o);
+    }
+  }
+#pragma unroll 1
+  for (int pc = 0; pc < stored; ++pc) {
+    uint32_t pp[16];
+    tmem_ld16(tS + pc * 16, pp);
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
+    tmem_st16(tS + pc * 16, pp);
+  }
+}
+
+// The diagonal tile, once per row-block and out of the hot loop: the scores of the keys after a row's own position
+// are set to -infinity in TMEM before the common path reads them.  Called by whole warps.
+static __device__ __noinline__ void mask_diag_tmem(uint32_t tS, int row) {
+#pragma unroll 1
+  for (int c = 0; c < BLK / 32; ++c) {
+    uint32_t sc[32];
+    tmem_ld32(tS + c * 32, sc);
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+      if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
+    tmem_st32(tS + c * 32, sc);
+  }
+  tmem_wait_st();
+}
+
+// kTrace: the phase trace compiled in (a profiling aid; its code in the hot loops costs a few per cent).
+template <bool kTrace>
 __global__ void __launch_bounds__(kThreadsPair, 1)
 attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v) {
@@ -205,7 +253,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   const int n_pairs = (a.Nb + 1) >> 1;
   const Abort ab{abort_flag, a.status};
   // Optional phase trace (one CTA, one thread per role): {(event << 32) | step, SM clock} pairs.
-  const bool tracing = a.trace != nullptr && blockIdx.x == 0;
+  const bool tracing = kTrace && a.trace != nullptr && blockIdx.x == 0;
   int trace_n = 0;
   auto trace = [&](int role, int event, int step) {
     if (tracing && trace_n < a.trace_cap) {
@@ -257,73 +305,71 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   };
 
   if (warp >= 8) {
-    if (warp == 10) {
-      // ---------------------------------------------------------- scheduler
-      // Takes the next position of the work order from the launch's counter, resolves it to (head, pair, list,
-      // counts) and posts it one item ahead of the roles that consume it.  Work order: the heads of one KV head
-      // together (their K/V set, 64 MB at 128K, stays in L2 while they run), inside such a group the longest
-      // row-block pairs first, heads fastest.
+    if (warp == 9) {
+      // ---------------------------------------------------------- producer
       const int n_items = a.n_heads * n_pairs;
       const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
-      for (int k = 0;; ++k) {
-        const int sl = k & 1;
-        if (k >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_EMPTY + sl), ((uint32_t)(k >> 1) & 1u) ^ 1u, ab, 40)))
-          break;
-        int id = -1;
-        if (lane == 0) {
-          int raw = poisoned ? n_items : atomicAdd(a.work_counter, 1);
-          Item it;
-          it.id = -1; it.slot = 0; it.u = 0; it.h = 0; it.list = -1; it.cntA = 0; it.cntB = 0;
-          if (raw < n_items) {
-            int rest = raw, g = 0;
-            while (g + 1 < a.n_groups && rest >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
-              rest -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
-              ++g;
-            }
-            const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
-            it.id = raw;
-            it.slot = a.order.v[a.group_start.v[g] + rest % ng];
-            it.u = n_pairs - 1 - rest / ng;
-            it.h = a.heads.v[it.slot];
-            it.list = a.lists_dev ? a.lists_dev[it.slot] : a.lists.v[it.slot];   // decided on the device, or by the host
-            if (it.list < 0) it.list = -1;
-            int cnt[2];
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-              const int i = 2 * it.u + x;
-              int c = 0;
-              if (i < a.Nb) {
-                c = it.list >= 0 ? a.counts[(size_t)it.list * a.Nb + i] : i + 1;
-                c = c < 0 ? 0 : (c > i + 1 ? i + 1 : c);
-              }
-              cnt[x] = c;
-            }
-            it.cntA = cnt[0];
-            it.cntB = cnt[1];
-          }
-          items[8 * sl + 0] = it.id;
-          items[8 * sl + 1] = it.slot;
-          items[8 * sl + 2] = it.u;
-          items[8 * sl + 3] = it.h;
-          items[8 * sl + 4] = it.list;
-          items[8 * sl + 5] = it.cntA;
-          items[8 * sl + 6] = it.cntB;
-          mbar_arrive(bar(BAR_ITEM_FULL + sl));
-          id = it.id;
-        }
-        id = __shfl_sync(0xffffffffu, id, 0);
-        if (id < 0) break;
-      }
-    } else if (warp == 9) {
-      // ---------------------------------------------------------- producer
       int gk = 0;        // merged key-blocks of the finished items (ring position of the next item's first)
       int issued_k = 0, issued_v = 0;   // K and V loads issued so far
       int relays = 0;    // relays to the issuing warp so far
       int qn = 0;        // items with work so far (Q loads)
       bool ok = true;
       for (int k = 0; ok; ++k) {
+        // Scheduling: the next position of the work order comes from the launch's counter; lane 0 resolves it to
+        // (head, pair, list, counts) and posts it for the other roles.  Work order: the heads of one KV head together
+        // (their K/V set, 64 MB at 128K, stays in L2 while they run), inside such a group the longest row-block pairs
+        // first, heads fastest.  The slot is free once the nine reader warps have taken the item two before this one.
         Item it;
-        if (!take_item(k, it, 14)) { ok = false; break; }
+        {
+          const int sl = k & 1;
+          if (k >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_EMPTY + sl), ((uint32_t)(k >> 1) & 1u) ^ 1u, ab, 40));
+          if (!ok) break;
+          it.id = -1; it.slot = 0; it.u = 0; it.h = 0; it.list = -1; it.cntA = 0; it.cntB = 0;
+          if (lane == 0) {
+            const int raw = poisoned ? n_items : atomicAdd(a.work_counter, 1);
+            if (raw < n_items) {
+              int rest = raw, g = 0;
+              while (g + 1 < a.n_groups && rest >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
+                rest -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
+                ++g;
+              }
+              const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
+              it.id = raw;
+              it.slot = a.order.v[a.group_start.v[g] + rest % ng];
+              it.u = n_pairs - 1 - rest / ng;
+              it.h = a.heads.v[it.slot];
+              it.list = a.lists_dev ? a.lists_dev[it.slot] : a.lists.v[it.slot];
+              if (it.list < 0) it.list = -1;
+              int cnt[2];
+#pragma unroll
+              for (int x = 0; x < 2; ++x) {
+                const int i = 2 * it.u + x;
+                int c = 0;
+                if (i < a.Nb) {
+                  c = it.list >= 0 ? a.counts[(size_t)it.list * a.Nb + i] : i + 1;
+                  c = c < 0 ? 0 : (c > i + 1 ? i + 1 : c);
+                }
+                cnt[x] = c;
+              }
+              it.cntA = cnt[0];
+              it.cntB = cnt[1];
+            }
+            items[8 * sl + 0] = it.id;
+            items[8 * sl + 1] = it.slot;
+            items[8 * sl + 2] = it.u;
+            items[8 * sl + 3] = it.h;
+            items[8 * sl + 4] = it.list;
+            items[8 * sl + 5] = it.cntA;
+            items[8 * sl + 6] = it.cntB;
+            mbar_arrive(bar(BAR_ITEM_FULL + sl));
+          }
+          it.id = __shfl_sync(0xffffffffu, it.id, 0);
+          it.u = __shfl_sync(0xffffffffu, it.u, 0);
+          it.h = __shfl_sync(0xffffffffu, it.h, 0);
+          it.list = __shfl_sync(0xffffffffu, it.list, 0);
+          it.cntA = __shfl_sync(0xffffffffu, it.cntA, 0);
+          it.cntB = __shfl_sync(0xffffffffu, it.cntB, 0);
+        }
         if (it.id < 0) break;
         const int cntA = it.cntA, cntB = it.cntB;
         if (cntA + cntB == 0) continue;
@@ -590,15 +636,10 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         // Then the max of chunks 2 and 3 is taken, and a move they ask for is made, BEFORE the first half of P is
         // handed over: after that no reference can move in this key-block, so the PV of keys 0..63 may run while
         // keys 64..127 are exponentiated from the registers they already sit in.
-        const bool diag = j == i;
         float tile_sum = 0.f;
         uint32_t sa[32], sb[32];
+        if (j == i) mask_diag_tmem(tS, row);
         tmem_ld32_async(tS, sa);
-        auto mask_diag = [&](uint32_t* sc, const int c) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (c * 32 + e > row) sc[e] = __float_as_uint(-CUDART_INF_F);
-        };
         auto chunk_max = [&](const uint32_t* sc) {
           float mx0 = max3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
           float mx1 = max3(__uint_as_float(sc[3]), __uint_as_float(sc[4]), __uint_as_float(sc[5]));
@@ -622,28 +663,9 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
             const float m_new = (mx > m_ref + 8.f) ? mx : m_ref;
             const float alpha = ex2_approx(m_ref - m_new);
-            if (t > 0) {
-              // O of the previous steps is relative to the old reference: bring it to the new one.
-              // (S of this step is complete, so the PV of the previous step, issued before it, is too.)
-#pragma unroll 1
-              for (int oc = 0; oc < D / 32; ++oc) {
-                uint32_t o[32];
-                tmem_ld32(tO + oc * 32, o);
-#pragma unroll
-                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                tmem_st32(tO + oc * 32, o);
-              }
-            }
-            // the P chunks of this key-block that are already stored (none of them handed over yet)
-#pragma unroll 1
-            for (int pc = 0; pc < stored; ++pc) {
-              uint32_t pp[16];
-              tmem_ld16(tS + pc * 16, pp);
-#pragma unroll
-              for (int e = 0; e < 16; ++e)
-                pp[e] = cvt_bf16x2(__uint_as_float(pp[e] << 16) * alpha, __uint_as_float(pp[e] & 0xffff0000u) * alpha);
-              tmem_st16(tS + pc * 16, pp);
-            }
+            // O of the previous steps is relative to the old reference (S of this step is complete, so the PV of
+            // the previous step, issued before it, is too); none of the stored P chunks has been handed over yet
+            rescale_tmem(tO, tS, alpha, stored, t > 0);
             l *= alpha;
             tile_sum *= alpha;
             m_ref = m_new;
@@ -672,23 +694,19 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         tmem_ld_wait();
         reg_fence32(sa);
         tmem_ld32_async(tS + 32, sb);
-        if (diag) mask_diag(sa, 0);
         move_reference(chunk_max(sa) * scale, 0);
         chunk_exps(sa, 0);
         tmem_ld_wait();
         reg_fence32(sb);
         tmem_ld32_async(tS + 64, sa);
-        if (diag) mask_diag(sb, 1);
         move_reference(chunk_max(sb) * scale, 1);
         chunk_exps(sb, 1);
         tmem_ld_wait();
         reg_fence32(sa);
         tmem_ld32_async(tS + 96, sb);
-        if (diag) mask_diag(sa, 2);
         float mx23 = chunk_max(sa);
         tmem_ld_wait();
         reg_fence32(sb);
-        if (diag) mask_diag(sb, 3);
         mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
         move_reference(mx23, 2);
         tmem_wait_st();
@@ -833,12 +851,13 @@ cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
       !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK) ||
       !make_map(&tv, a.v, a.v_sh, a.v_sn, a.n_kv_heads, a.N, D, BLK))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
+  auto kernel = a.trace ? attn_pair_kernel<true> : attn_pair_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
   if (e != cudaSuccess) return e;
   // Persistent CTAs, one per SM, take the items of the work order from a counter that starts at zero.
   e = cudaMemsetAsync(a.work_counter, 0, sizeof(int), s);
   if (e != cudaSuccess) return e;
-  attn_pair_kernel<<<attn_pair_ctas(a.n_heads, a.Nb), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
+  kernel<<<attn_pair_ctas(a.n_heads, a.Nb), kThreadsPair, kSmemTotal, s>>>(a, tq, tk, tv);
   return cudaGetLastError();
 }
 

@@ -46,17 +46,18 @@ struct Abort {
 // The checks are kept off the fast path: the CTA's own abort flag (shared memory) every 64
 // polls, the time limit and the global status word (a trip to L2 that would delay the wake-up
 // by hundreds of cycles if it were made often) every 4096.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where,
-                                          long long limit_cycles = kWaitCycles) {
-  if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is out of line: inlined at every wait it made the kernels' hot loops large enough to cost
+// several per cent (instruction fetch), and a wait that does not succeed at once has time for a call.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* flag, int* status, int where,
+                                            long long limit_cycles) {
   long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
-      if (*ab.flag) return false;
+      if (*flag) return false;
       if ((it & 4095u) == 0u) {
-        if (*reinterpret_cast<volatile int*>(ab.status) != 0) {   // another CTA already gave up
-          *ab.flag = 1;
+        if (*reinterpret_cast<volatile int*>(status) != 0) {   // another CTA already gave up
+          *flag = 1;
           return false;
         }
         const long long now = clock64();
@@ -65,9 +66,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
       }
     }
   }
-  *ab.flag = 1;
-  if (atomicCAS(ab.status, 0, (int)SP_ERR_TIMEOUT) == 0) ab.status[1] = where;
+  *flag = 1;
+  if (atomicCAS(status, 0, (int)SP_ERR_TIMEOUT) == 0) status[1] = where;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int where,
+                                          long long limit_cycles = kWaitCycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, ab.flag, ab.status, where, limit_cycles);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
