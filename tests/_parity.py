@@ -108,3 +108,94 @@ def check_layer(L, gamma, out, mask, row_blocks=None):
     return worst, exempt
 
 
+
+
+# ------------------------------------------------------------------ sampled check of a layer at several thresholds
+
+def sample_rows(Nb, n, seed):
+    """Row-blocks 0, 1, Nb/2, Nb-1 and seeded others, n in all (all of them when Nb <= n)."""
+    fixed = {0, min(1, Nb - 1), Nb // 2, Nb - 1}
+    rng = np.random.default_rng(seed)
+    rest = [int(i) for i in rng.permutation(Nb) if int(i) not in fixed]
+    return sorted(fixed | set(rest[:max(0, n - len(fixed))]))
+
+
+def check_layer_sampled(L, runs, rows, members=None, what=""):
+    """Sampled row-blocks of one layer against the oracle, at one or several thresholds.
+
+    runs: {gamma: (out [Hq, N, d] tensor, mask [Hq, Nb, Nb] tensor)} as sp_prefill_attn returned them on the SAME inputs.
+    rows: row-blocks to check (a row-block's mask and outputs depend only on its own queries and the keys before it).
+    members: {gamma: non-pivot heads whose outputs are checked}; default: all of them at every gamma.
+    The pivots' dense attention and importance rows do not depend on gamma, so the oracle computes them once per
+    (pivot, row-block) and cuts them at every gamma.  Mask rule: bit-exact, except row-blocks whose oracle cumulative
+    mass at the cut, or just before it, is within MASK_BAND of gamma; those are counted (and returned), and outputs of
+    heads that use such a row are not compared there.  Returns dict(worst_max_abs, worst_rel_l2, exempt, near_ties).
+    """
+    cfg = L["cfg"]
+    B, Nb, Hq, Hkv = cfg.block, cfg.seq // cfg.block, cfg.n_q_heads, cfg.n_kv_heads
+    piv = list(L["pivot_heads"])
+    src, mask_src = orc.share_masks(L["cluster_map"], piv)
+    kv = {}
+
+    def kvf(g):
+        if g not in kv:
+            kv[g] = (f64(L["k"][g]), f64(L["v"][g]))
+        return kv[g]
+
+    masks = {g_: m.cpu().numpy() for g_, (_, m) in runs.items()}
+    causal = np.tril(np.ones((Nb, Nb), np.uint8))
+    stats = {"worst_max_abs": 0.0, "worst_rel_l2": 0.0, "exempt": 0, "near_ties": 0, "rows": len(rows)}
+    clean = {g_: {} for g_ in runs}          # gamma -> pivot slot -> set of row-blocks whose mask agreed
+    ref_rows = {g_: {} for g_ in runs}       # gamma -> (pivot slot, row-block) -> oracle mask row
+    for t, p in enumerate(piv):
+        Qp = f64(L["q"][p])
+        Kg, Vg = kvf(orc.kv_head_of(p, Hq, Hkv))
+        for g_ in runs:
+            clean[g_][t] = set()
+        for i in rows:
+            o_ref, mass = orc.attention_rowblock(Qp, Kg, Vg, i, B)
+            for g_, (out, _) in runs.items():
+                got = f64(out[p, i * B:(i + 1) * B])
+                ma, rl = out_errors(got, o_ref)
+                assert ma <= OUT_MAX_ABS and rl <= OUT_REL_L2, f"{what} pivot {p} row-block {i} gamma {g_}: {ma:.3e} {rl:.3e}"
+                stats["worst_max_abs"] = max(stats["worst_max_abs"], ma)
+                stats["worst_rel_l2"] = max(stats["worst_rel_l2"], rl)
+                gam = gamma32(g_)
+                sel, info = orc.block_mask_row(mass, i, gam)
+                ref_row = np.zeros(Nb, np.uint8)
+                ref_row[:i + 1] = sel
+                ref_rows[g_][(t, i)] = ref_row
+                if info["tie_gap"] <= MASK_BAND:
+                    stats["near_ties"] += 1
+                if np.array_equal(masks[g_][p, i], ref_row):
+                    clean[g_][t].add(i)
+                else:
+                    near = abs(info["cum_at_cut"] - gam) <= MASK_BAND or abs(info["cum_before_cut"] - gam) <= MASK_BAND
+                    assert near, (f"{what} pivot {p} row-block {i} gamma {g_}: mask differs away from the threshold "
+                                  f"(cum {info['cum_before_cut']:.9f} -> {info['cum_at_cut']:.9f})")
+                    stats["exempt"] += 1
+        del Qp
+    for g_, (out, _) in runs.items():
+        m = masks[g_]
+        hs = [h for h in range(Hq) if h not in piv] if members is None else list(members[g_])
+        for h in range(Hq):                       # reported patterns: integer work, every head
+            if mask_src[h] >= 0:
+                assert np.array_equal(m[h][rows], m[piv[mask_src[h]]][rows])
+            else:
+                assert np.array_equal(m[h][rows], causal[rows])
+            assert np.all(np.triu(m[h], 1) == 0)
+        for h in hs:
+            Qh = f64(L["q"][h])
+            Kg, Vg = kvf(orc.kv_head_of(h, Hq, Hkv))
+            for i in rows:
+                if src[h] >= 0:
+                    if i not in clean[g_][src[h]]:
+                        continue                  # row-block whose mask legitimately flipped
+                    o_ref, _ = orc.attention_rowblock(Qh, Kg, Vg, i, B, mask_row=ref_rows[g_][(src[h], i)])
+                else:
+                    o_ref, _ = orc.attention_rowblock(Qh, Kg, Vg, i, B)
+                ma, rl = out_errors(f64(out[h, i * B:(i + 1) * B]), o_ref)
+                assert ma <= OUT_MAX_ABS and rl <= OUT_REL_L2, f"{what} head {h} row-block {i} gamma {g_}: {ma:.3e} {rl:.3e}"
+                stats["worst_max_abs"] = max(stats["worst_max_abs"], ma)
+                stats["worst_rel_l2"] = max(stats["worst_rel_l2"], rl)
+    return stats

@@ -36,6 +36,35 @@ def _oracle_cut(At, g):
     return res, cum_at.reshape(Nb, Nb), flat.reshape(Nb, Nb)
 
 
+def _mask_differences_in_band(m, res, cum_at, flat, g, band=None):
+    """Entries where the GPU mask m differs from the oracle's: each must lie in the band (the oracle's cumulative
+    normalised score with it, or just before it, within `band` of gamma).  One more case follows from such a flip: a
+    row-block whose selection is empty on one side only receives its diagonal there, so a differing diagonal is
+    accepted when one side's row is the diagonal alone and every other differing entry of the row is in the band.
+    Returns the number of differing entries (all accounted for)."""
+    band = SCORE_BAND if band is None else band
+    diff = np.argwhere(m != res["mask"])
+    near = {(int(i), int(j)): (abs(cum_at[i, j] - g) <= band or abs(cum_at[i, j] - flat[i, j] - g) <= band) for i, j in diff}
+    for (i, j), ok in near.items():
+        if ok:
+            continue
+        others = [e for e in near if e[0] == i and e != (i, j)]
+        alone = (m[i].sum() == 1 and m[i, i] == 1) or (res["mask"][i].sum() == 1 and res["mask"][i, i] == 1)
+        assert j == i and alone and others and all(near[e] for e in others), \
+            f"block ({i}, {j}) differs away from the cut: cumulative {cum_at[i, j]:.9f}, gamma {g:.9f}"
+    return len(diff)
+
+
+def _lines_differences_in_band(got, want, a, g, band=None):
+    """Selected lines (key columns or offsets) against the oracle's: a line may differ only inside the band."""
+    band = VS_BAND if band is None else band
+    cum, f = _cum_at(a, g)
+    diff = np.flatnonzero(got.astype(bool) != want)
+    for e in diff:
+        assert abs(cum[e] - g) <= band or abs(cum[e] - f[e] - g) <= band, (int(e), float(cum[e]), g)
+    return len(diff)
+
+
 @pytest.mark.parametrize("name,seq,gamma", [("llama8b_32k", 4096, 0.9), ("tiny", 2048, 0.8), ("qwen7b_64k", 4096, 0.95)])
 def test_pooled_logits_and_pattern_match_oracle(binding, name, seq, gamma):
     L = synth.make_layer(synth.scaled(synth.CONFIGS[name], seq), seed=3)
@@ -66,13 +95,9 @@ def test_pooled_logits_and_pattern_match_oracle(binding, name, seq, gamma):
         np.testing.assert_allclose(last[t].cpu().numpy(), res["a_last"], rtol=0, atol=1e-6)
         m = mask[t].cpu().numpy()
         assert np.all(m[~tri] == 0) and np.all(m.sum(axis=1) >= 1)
-        # entries may differ from the oracle only next to the cut (or as a forced diagonal that follows from it)
-        diff = np.argwhere(m != res["mask"])
-        for i, j in diff:
-            near = abs(cum_at[i, j] - g) <= SCORE_BAND or abs(cum_at[i, j] - flat[i, j] - g) <= SCORE_BAND
-            forced = i == j and (m[i].sum() == 1 or res["mask"][i].sum() == 1)
-            assert near or forced, (h, i, j, cum_at[i, j], g)
-        assert len(diff) <= 4
+        n_diff = _mask_differences_in_band(m, res, cum_at, flat, g)
+        if n_diff:
+            print(f"{name} head {h}: {n_diff} blocks inside the {SCORE_BAND} band flipped")
         # lists and counts describe the mask
         c, ix = counts[t].cpu().numpy(), idx[t].cpu().numpy()
         for i in range(Nb):
@@ -192,11 +217,9 @@ def test_vertical_slash_pattern_matches_oracle(binding, name, seq, gamma):
     for t, h in enumerate(heads):
         res = ppo.search_vertical_slash_pattern(Q[h], K[h // G], g, B)
         for got, want, a in ((sv[t].cpu().numpy(), res["sel_v"], res["a_v"]), (ss[t].cpu().numpy(), res["sel_s"], res["a_s"])):
-            cum, f = _cum_at(a, g)
-            diff = np.flatnonzero(got.astype(bool) != want)
-            for e in diff:
-                assert abs(cum[e] - g) <= VS_BAND or abs(cum[e] - f[e] - g) <= VS_BAND, (h, e, cum[e], g)
-            assert len(diff) <= 4
+            n_diff = _lines_differences_in_band(got, want, a, g)
+            if n_diff:
+                print(f"{name} head {h}: {n_diff} lines inside the {VS_BAND} band flipped")
         m = mask[t].cpu().numpy()
         # the mask is exactly what the GPU's own selected lines imply (integer work: bit-exact)
         gv, gs = sv[t].cpu().numpy().astype(bool), ss[t].cpu().numpy().astype(bool)
@@ -410,12 +433,13 @@ def test_layers_with_cross_layer_dictionary(binding, pooled):
                 stored[r[2]] = mask_h[h].copy()
                 # the stored pattern is what the construction call gives for this head
                 if pooled:
-                    res = ppo.construct_pivotal_pattern(ppo.pooled_logits(Q[h], K[h // G], B), par.gamma32(gamma))
-                    assert (mask_h[h] != res["mask"]).sum() <= 4
+                    res, cum_at, flat = _oracle_cut(ppo.pooled_logits(Q[h], K[h // G], B), par.gamma32(gamma))
+                    _mask_differences_in_band(mask_h[h], res, cum_at, flat, par.gamma32(gamma))
                 else:
                     I, _ = orc.importance_map(Q, K, V, h, B)
-                    M, _, _, _ = orc.block_mask_from_importance(I, par.gamma32(gamma))
-                    assert (mask_h[h] != M).sum() <= 2
+                    M, _, _, infos = orc.block_mask_from_importance(I, par.gamma32(gamma))
+                    bad, _ = par.compare_mask_rows(mask_h[h], M, infos, par.gamma32(gamma), range(Nb))
+                    assert bad == 0, f"layer {li} pivot {h}: {bad} row-blocks differ outside the {par.MASK_BAND} band"
             elif r[0] == "vs":
                 assert pat_h[h] == 2
             else:
@@ -440,6 +464,161 @@ def test_layers_with_cross_layer_dictionary(binding, pooled):
     assert cross_layer > 0                                               # a pattern stored by one layer is reused by a later one
     d.clear()
     assert d.count() == 0
+
+
+# ------------------------------------------------------------------ the same calls at the sizes the benchmark times
+
+def _lines_mask(gv, gs, Nb, B, N):
+    """index_to_mask of "Search Vertical Slash Pattern" from selected columns gv and offsets gs (vectorised restatement
+    of the rule the small-size test spells out entry by entry): block (i, j), j <= i, is on if key-block j holds a
+    selected column or a selected offset lies in [(i-j)B-(B-1), (i-j)B+(B-1)]; an empty row gets its diagonal."""
+    colb = gv.reshape(Nb, B).any(axis=1)
+    pre = np.concatenate([[0], np.cumsum(gs.astype(np.int64))])
+    by_delta = np.zeros(Nb, bool)
+    for dlt in range(Nb):
+        lo, hi = max(dlt * B - (B - 1), 0), min(dlt * B + (B - 1), N - 1)
+        by_delta[dlt] = pre[hi + 1] - pre[lo] > 0
+    i_, j_ = np.meshgrid(np.arange(Nb), np.arange(Nb), indexing="ij")
+    want = (j_ <= i_) & (colb[None, :] | by_delta[np.clip(i_ - j_, 0, Nb - 1)])
+    want = want.astype(np.uint8)
+    for i in np.flatnonzero(want.sum(axis=1) == 0):
+        want[i, i] = 1
+    return want
+
+
+def test_decision_and_vertical_slash_at_131072_tokens(binding):
+    """Algorithms "Determine Sparse Pattern" and "Search Vertical Slash Pattern" on the benchmark's 131072-token
+    layer (Nb = 1024: 131072-entry cuts, 128 sweep chunks per head)."""
+    from oracle import shareprefill_oracle as orc
+    cfg = synth.CONFIGS["llama8b_128k"]
+    L = synth.make_layer(cfg, seed=0, device="cuda")
+    B, Nb, N, Hq = cfg.block, cfg.seq // cfg.block, cfg.seq, cfg.n_q_heads
+    G = Hq // cfg.n_kv_heads
+    piv = list(L["pivot_heads"])
+    ctx = binding.Context()
+    q, k, v = L["q"], L["k"], L["v"]
+    Lh = dict(L, q=q.cpu(), k=k.cpu(), v=v.cpu())
+    kv64 = {}
+
+    def K64(g):
+        if g not in kv64:
+            kv64[g] = par.f64(Lh["k"][g])
+        return kv64[g]
+
+    # ---- decision: every head against the representative of its cluster's pivot (the pivot's own a^)
+    first = {}
+    for t, p in enumerate(piv):
+        first.setdefault(L["cluster_map"][p], t)
+    heads = list(range(Hq))
+    rows = [first.get(L["cluster_map"][h], -1) for h in heads]
+    a_hat = [ppo.last_block_distribution(par.f64(Lh["q"][h]), K64(h // G), B) for h in heads]
+    ref = [ppo.determine_pattern(a_hat[h], a_hat[piv[r]] if r >= 0 else None, 0.3, 0.2) for h, r in zip(heads, rows)]
+    def widest_gap(values):                                     # a threshold that splits the heads and is close to few of them
+        w = np.sort(np.asarray(values))
+        w = w[len(w) // 5: len(w) - len(w) // 5 + 1]
+        gi = int(np.argmax(w[1:] - w[:-1]))
+        return float(0.5 * (w[gi] + w[gi + 1]))
+
+    delta = widest_gap([r[1] for r in ref])
+    tau = widest_gap([r[2] for r in ref if np.isfinite(r[2]) and r[2] > 0])
+    a_tilde = torch.from_numpy(np.stack([a_hat[p] for p in piv]).astype(np.float32)).cuda()
+    pat = torch.full((Hq,), -1, dtype=torch.int32, device="cuda")
+    dist = torch.full((Hq, 2), float("nan"), device="cuda")
+    ctx.sp_determine_pattern(q, k, heads, B, a_tilde, rows, delta, tau, pat, dist_out=dist)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    got_p, got_d = pat.cpu().numpy(), dist.cpu().numpy()
+    checked = 0
+    for x, (h, r) in enumerate(zip(heads, rows)):
+        _, ds, dm = ref[x]
+        assert float(got_d[x, 0]) ** 2 == pytest.approx(ds * ds, abs=DIV_ATOL), (h, got_d[x, 0], ds)
+        assert float(got_d[x, 1]) ** 2 == pytest.approx(dm * dm, abs=DIV_ATOL), (h, got_d[x, 1], dm)
+        if min(abs(ds - delta), abs(dm - tau)) > DIST_MARGIN:
+            assert got_p[x] == (0 if (ds < delta and dm < tau) else 1), (h, ds, dm, delta, tau)
+            checked += 1
+    assert checked >= Hq // 4 and 0 < int((got_p == 0).sum()) < Hq
+    print(f"decision at 131072 tokens: {checked} of {Hq} decisions clear of the thresholds by {DIST_MARGIN}; d_sparse "
+          f"{min(r[1] for r in ref):.4f}..{max(r[1] for r in ref):.4f}, delta {delta:.4f}, tau {tau:.4f}, "
+          f"max |d^2 error| {max(abs(float(got_d[x, 0]) ** 2 - ref[x][1] ** 2) for x in range(Hq)):.1e}")
+
+    # ---- vertical-slash search for three heads; the third one's lists then drive the block-sparse kernel
+    vs_heads = [1, Hq - 1, 0]
+    gamma = 0.9
+    g = par.gamma32(gamma)
+    mask = torch.full((3, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+    counts = torch.full((3, Nb), -5, dtype=torch.int32, device="cuda")
+    idx = torch.full((3, Nb, Nb), -5, dtype=torch.int32, device="cuda")
+    sv = torch.full((3, N), 9, dtype=torch.uint8, device="cuda")
+    ss = torch.full((3, N), 9, dtype=torch.uint8, device="cuda")
+    ctx.sp_vertical_slash_pattern(q, k, vs_heads, gamma, B, mask, counts, idx, sel_v_out=sv, sel_s_out=ss)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    flipped = 0
+    for t, h in enumerate(vs_heads):
+        a_v, a_s = ppo.vertical_slash_scores(par.f64(Lh["q"][h]), K64(h // G), B)
+        sel_v, _ = ppo.cumulative_select(a_v, g)
+        sel_s, _ = ppo.cumulative_select(a_s, g)
+        gv, gs = sv[t].cpu().numpy().astype(bool), ss[t].cpu().numpy().astype(bool)
+        flipped += _lines_differences_in_band(gv, sel_v, a_v, g) + _lines_differences_in_band(gs, sel_s, a_s, g)
+        m = mask[t].cpu().numpy()
+        assert np.array_equal(m, _lines_mask(gv, gs, Nb, B, N))            # integer work: bit-exact on the GPU's own lines
+        c, ix = counts[t].cpu().numpy(), idx[t].cpu().numpy()
+        assert np.array_equal(c, m.sum(axis=1))
+        for i in (0, 1, Nb // 2, Nb - 1):
+            sel = np.flatnonzero(m[i])
+            assert np.array_equal(ix[i, :c[i]], sel) and np.all(ix[i, c[i]:] == -1)
+    print(f"vertical-slash at 131072 tokens: {flipped} lines inside the {VS_BAND} band flipped; mask densities "
+          f"{[round(float(mask[t].sum()) / (Nb * (Nb + 1) / 2), 3) for t in range(3)]}")
+    out = torch.full_like(q, float("nan"))
+    ctx.sp_block_sparse_attn(q, k, v, vs_heads[:1], [0], counts, idx, B, out)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    h = vs_heads[0]
+    m0 = mask[0].cpu().numpy()
+    Qh, Kg, Vg = par.f64(Lh["q"][h]), K64(h // G), par.f64(Lh["v"][h // G])
+    for i in par.sample_rows(Nb, 6, 5):
+        o_ref, _ = orc.attention_rowblock(Qh, Kg, Vg, i, B, mask_row=m0[i])
+        par.assert_out_close(par.f64(out[h, i * B:(i + 1) * B]), o_ref, f"head {h} row-block {i}")
+
+
+@pytest.mark.parametrize("name,gamma", [("llama8b_32k", 0.9), ("llama8b_128k", 0.9)])
+def test_pooled_construction_at_full_size(binding, name, gamma):
+    """Algorithm "Construct Pivotal Pattern" as the paper writes it, one pivot of the 32768- and of the 131072-token
+    workload in full: the pooled map, the global cut on the library's own map, and the global cut fed with the
+    oracle's map (so that the cut's fixed-point sums are checked at 32896 and 524800 scores by themselves)."""
+    cfg = synth.CONFIGS[name]
+    L = synth.make_layer(cfg, seed=0, device="cuda")
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    h = L["pivot_heads"][0]
+    ctx = binding.Context()
+    pooled = torch.full((1, Nb, Nb), float("nan"), device="cuda")
+    ctx.sp_pooled_logits(L["q"], L["k"], [h], B, pooled)
+    torch.cuda.synchronize()
+    At = ppo.pooled_logits(par.f64(L["q"][h].cpu()), par.f64(L["k"][h // G].cpu()), B)
+    tri = np.tril(np.ones((Nb, Nb), bool))
+    got = pooled[0].cpu().numpy().astype(np.float64)
+    assert np.all(got[~tri] == -np.inf)
+    err = float(np.abs(got[tri] - At[tri]).max())
+    assert err <= POOLED_ATOL, err
+    g = par.gamma32(gamma)
+    res, cum_at, flat = _oracle_cut(At, g)
+    n_diff = {}
+    for label, src in (("own map", pooled), ("oracle's map", torch.from_numpy(At[None].astype(np.float32)).cuda())):
+        mask = torch.full((1, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+        counts = torch.full((1, Nb), -5, dtype=torch.int32, device="cuda")
+        idx = torch.full((1, Nb, Nb), -5, dtype=torch.int32, device="cuda")
+        last = torch.full((1, Nb), float("nan"), device="cuda")
+        ctx.sp_pattern_from_pooled(src, gamma, mask, counts, idx, last_row_out=last)
+        torch.cuda.synchronize()
+        assert ctx.status() == (0, 0)
+        m = mask[0].cpu().numpy()
+        assert np.all(m[~tri] == 0) and np.all(m.sum(axis=1) >= 1)
+        n_diff[label] = _mask_differences_in_band(m, res, cum_at, flat, g)
+        np.testing.assert_allclose(last[0].cpu().numpy(), res["a_last"], rtol=0, atol=1e-6)
+        assert np.array_equal(counts[0].cpu().numpy(), m.sum(axis=1))
+    print(f"{name} pivot {h}: pooled map max error {err:.2e}; blocks inside the {SCORE_BAND} band that flipped: {n_diff}; "
+          f"density {float(res['mask'].sum()) / tri.sum():.4f}")
 
 
 # ------------------------------------------------------------------ argument checking of these calls (host side)
