@@ -38,13 +38,27 @@ if ROOT not in sys.path:
 
 from paper_2505_19578_b200 import synth  # noqa: E402
 
-# DRAM bytes (read + write) per launch of the attention kernel from an ncu capture of this very workload
-# (profiles/attn_pair_kernel_llama8b_128k_dram_traffic.md); valid for the default workload, gamma and seed only,
-# and to be set back to None whenever the attention kernel changes.
-NCU_DRAM_TRAFFIC = {
-    ("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 1970131456 + 1190532096,
-    ("llama8b_128k", 131072, 0.9, 0, "block_sparse_attn"): 1485898496 + 903549440,
-}
+# DRAM bytes (read + write) per launch of the attention kernel, from ncu captures: a small tracked table
+# (one line per workload / length / gamma / seed / call, with the command that produced it in its header).  A
+# workload without a line, or a line taken before the kernel last changed (removed then), gives null.
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "attention_kernel_dram_traffic.txt")
+
+
+def load_traffic_table(path=TRAFFIC_TABLE):
+    """{(workload, seq, gamma, seed, call): bytes per launch}; lines starting with # are comments."""
+    table = {}
+    if not os.path.exists(path):
+        return table
+    for line in open(path):
+        line = line.split("#", 1)[0].strip()
+        if not line:
+            continue
+        f = line.split()
+        if len(f) != 6:
+            continue
+        table[(f[0], int(f[1]), round(float(f[2]), 6), int(f[3]), f[4])] = int(f[5])
+    return table
+
 
 METRIC = "effective_tflops_prefill_attention_layer"
 UNIT = "TFLOP/s"
@@ -162,6 +176,86 @@ def oracle_sample_time(L, gamma, row_blocks):
     except Exception:
         threads = os.cpu_count() or 1
     return dt, flops, threads
+
+
+def time_config(binding, ctx, L, gamma, steps, stream, dense=True):
+    """Per-kernel times of one layer on workload L at `gamma`: the three public calls with CUDA events between them,
+    one warm-up, `steps` timed; the build's own dense kernel on every head beside it.  Compact dict for the
+    other_configs block."""
+    cfg = L["cfg"]
+    q, k, v, cm, piv = L["q"], L["k"], L["v"], L["cluster_map"], L["pivot_heads"]
+    B, Nb = cfg.block, cfg.seq // cfg.block
+    dev = q.device
+    out = torch.empty_like(q)
+    members = [h for h in range(cfg.n_q_heads) if h not in piv]
+    first_pivot_of = {}
+    for t, p in enumerate(piv):
+        first_pivot_of.setdefault(cm[p], t)
+    lists = [first_pivot_of.get(cm[h], -1) if cm[h] >= 0 else -1 for h in members]
+    imp = torch.empty(len(piv), Nb, Nb, device=dev)
+    pm = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device=dev)
+    counts = torch.empty(len(piv), Nb, dtype=torch.int32, device=dev)
+    indices = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device=dev)
+
+    def split_step(e):
+        e[0].record(stream)
+        ctx.sp_dense_pivot_attn(q, k, v, piv, B, out, importance_out=imp, stream=stream)
+        e[1].record(stream)
+        ctx.sp_block_mask_from_importance(imp, gamma, pm, counts, indices, stream=stream)
+        e[2].record(stream)
+        ctx.sp_block_sparse_attn(q, k, v, members, lists, counts, indices, B, out, stream=stream)
+        e[3].record(stream)
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps + 1)]
+    sampler = ClockSampler(dev.index or 0)
+    split_step(ev[0])
+    torch.cuda.synchronize()
+    sampler.start()
+    for e in ev[1:]:
+        split_step(e)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    k1 = sum(e[0].elapsed_time(e[1]) for e in ev[1:]) / steps
+    k2 = sum(e[1].elapsed_time(e[2]) for e in ev[1:]) / steps
+    k3 = sum(e[2].elapsed_time(e[3]) for e in ev[1:]) / steps
+    # the whole call
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, B, out, stream=stream)
+    torch.cuda.synchronize()
+    w0.record(stream)
+    for _ in range(steps):
+        ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, B, out, stream=stream)
+    w1.record(stream)
+    torch.cuda.synchronize()
+    ms = w0.elapsed_time(w1) / steps
+    cnt = counts.cpu().numpy()
+    tiles_causal = Nb * (Nb + 1) // 2
+    pivot_tiles = len(piv) * tiles_causal
+    member_tiles = int(sum(int(cnt[l].sum()) if l >= 0 else tiles_causal for l in lists))
+    Ft = tile_flops(cfg)
+    dense_ms = None
+    if dense:
+        heads = list(range(cfg.n_q_heads))
+        ctx.sp_dense_pivot_attn(q, k, v, heads, B, out, stream=stream)
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(2):
+            ctx.sp_dense_pivot_attn(q, k, v, heads, B, out, stream=stream)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        dense_ms = d0.elapsed_time(d1) / 2
+    assert ctx.status() == (0, 0), "device-side wait timed out"
+    dens = [float(cnt[t].sum()) / tiles_causal for t in range(len(piv))]
+    return {
+        "workload": cfg.name, "seq": cfg.seq, "gamma": gamma, "n_pivots": len(piv), "steps": steps,
+        "ms_per_layer": ms, "kernels_ms": {"pivot_dense_attn": k1, "block_mask": k2, "block_sparse_attn": k3},
+        "visited_tflops": {"pivot_dense_attn": pivot_tiles * Ft / (k1 * 1e-3) / 1e12,
+                           "block_sparse_attn": member_tiles * Ft / (k3 * 1e-3) / 1e12 if k3 > 0 else 0.0},
+        "mask_density_min_max": [min(dens), max(dens)] if dens else None,
+        "dense_baseline_ms": dense_ms, "speedup_vs_dense": dense_ms / ms if dense_ms else None,
+        "clocks": {k_: clocks.get(k_) for k_ in ("sm_mhz", "sm_max_mhz", "reasons")},
+    }
 
 
 def workload_cfg(args):
@@ -304,6 +398,8 @@ def run_ours(args):
 
     # ---- optional: a stack of layers (each its own seeded inputs and 3-6 clusters), times summed over layers
     stack = None
+    if args.stack_layers is None:
+        args.stack_layers = 32 if (world == 1 and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9) else 0
     if rank == 0 and args.stack_layers > 0:
         import dataclasses
         import random
@@ -332,6 +428,20 @@ def run_ours(args):
                  "dense_ms": None if args.no_dense else t_dense,
                  "speedup_vs_dense": None if args.no_dense else t_dense / t_sparse,
                  "note": "every layer has its own seeded q, k, v and 3-6 clusters (one pivot each); layers treated independently"}
+
+    # ---- the other configurations named next to the default one: the gamma sweep on the same inputs, the 32K and the
+    #      GQA-7 64K layer (a few steps each; per-kernel times, visited-tile rates, dense, clocks)
+    others = None
+    if rank == 0 and not args.no_other_configs and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9:
+        others = []
+        n_other = max(2, min(args.steps, 5))
+        for g_ in (0.8, 0.95):
+            others.append(time_config(binding, ctx, L, g_, n_other, stream, dense=False))
+        for name in ("llama8b_32k", "qwen7b_64k"):
+            Lo = synth.make_layer(synth.CONFIGS[name], seed=args.seed, device=str(dev))
+            others.append(time_config(binding, ctx, Lo, 0.9, n_other, stream, dense=not args.no_dense))
+            del Lo
+            torch.cuda.empty_cache()
 
     # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
     literal = None
@@ -448,8 +558,8 @@ def run_ours(args):
         "frac": dom[2] / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
         "peak_kind": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
         "frac_of_burst_peak": dom[2] / peaks["bf16_tflops"],
-        "traffic": NCU_DRAM_TRAFFIC.get((cfg.name, cfg.seq, round(gamma, 6), args.seed, dom[0])),
-        "traffic_unit": "bytes of DRAM read + write per launch (ncu, same workload)",
+        "traffic": load_traffic_table().get((cfg.name, cfg.seq, round(gamma, 6), args.seed, dom[0])),
+        "traffic_unit": "bytes of DRAM read + write per launch (ncu, same workload; null: not taken since the kernel changed)",
         "ms_per_launch": dom[1], "flops_per_launch": (pivot_tiles if dom[0].startswith("pivot") else member_tiles) * Ft,
         "timing": "CUDA events around each of the three public calls, same inputs, same number of steps",
     }
@@ -480,6 +590,7 @@ def run_ours(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "paper_literal_pattern": literal,
         "layer_stack": stack,
+        "other_configs": others,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -509,8 +620,11 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
-    ap.add_argument("--stack-layers", type=int, default=0,
-                    help="also run a stack of this many independent layers (3-6 seeded clusters each) and sum their times")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the compact block on the other configurations (gamma 0.8 / 0.95, 32K, 64K GQA-7)")
+    ap.add_argument("--stack-layers", type=int, default=None,
+                    help="also run a stack of this many independent layers (3-6 seeded clusters each) and sum their "
+                         "times; default: 32 on the default 131072-token workload at N = 1, otherwise 0")
     ap.add_argument("--no-literal", action="store_true", help="skip the paper-literal pattern construction leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()

@@ -65,3 +65,12 @@ def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
     env1 = dict(os.environ, RANK="1", WORLD_SIZE="2")
     out1 = subprocess.run(cmd, capture_output=True, text=True, env=env1, timeout=600)
     assert out1.returncode == 0 and out1.stdout.strip() == ""
+
+
+def test_traffic_table_parsing(tmp_path):
+    import bench
+    p = tmp_path / "t.txt"
+    p.write_text("# comment\n\nllama8b_128k 131072 0.9 0 pivot_dense_attn 123456  # trailing note\nbad line\n")
+    t = bench.load_traffic_table(str(p))
+    assert t == {("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 123456}
+    assert bench.load_traffic_table(str(tmp_path / "missing.txt")) == {}
