@@ -443,6 +443,64 @@ def run_ours(args):
             del Lo
             torch.cuda.empty_cache()
 
+    # ---- a workload on which the paper's thresholds (gamma 0.9, delta 0.3, tau 0.2) decide something: two families
+    #      of heads, one sharing its pivots' patterns, one falling back to vertical-slash.  One layer through
+    #      sp_prefill_attn_auto, then a stack of layers through the cross-layer dictionary (pivots only where a cluster
+    #      has no pattern yet; later layers reuse what earlier ones stored)
+    mixed = None
+    if (rank == 0 and not args.no_mixed and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9):
+        mcfg = synth.CONFIGS["llama8b_128k_mixed"]
+        Lm = synth.make_layer(mcfg, seed=args.seed, device=str(dev))
+        mout = torch.empty_like(Lm["q"])
+        mpat = torch.empty(mcfg.n_q_heads, dtype=torch.int32, device=dev)
+        me = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for _ in range(2):
+            me[0].record(stream)
+            ctx.sp_prefill_attn_auto(Lm["q"], Lm["k"], Lm["v"], Lm["cluster_map"], Lm["pivot_heads"], gamma, 0.3, 0.2, B,
+                                     mout, pattern_out=mpat, stream=stream)
+            me[1].record(stream)
+            torch.cuda.synchronize()
+        mp = mpat.cpu().numpy()
+        mixed = {"workload": mcfg.name, "gamma": gamma, "delta": 0.3, "tau": 0.2,
+                 "prefill_attn_auto": {"ms_per_layer": me[0].elapsed_time(me[1]),
+                                       "heads_dense_shared_vslash": [int((mp == c).sum()) for c in (0, 1, 2)]}}
+        n_dict_layers = args.stack_layers if args.stack_layers > 0 else 0
+        if n_dict_layers:
+            pd = binding.PatternDict(ctx, mcfg.n_clusters, mcfg.n_q_heads, mcfg.seq, B)
+            t_layers, totals, new_pivots = 0.0, [0, 0, 0], []
+            for layer in range(n_dict_layers):
+                Ll = Lm if layer == 0 else synth.make_layer(mcfg, seed=args.seed + 1 + layer, device=str(dev),
+                                                            structure_seed=args.seed)
+                before = pd.count()
+                if layer == 0:                          # warm the kernels of this flow once, on a dictionary of its own
+                    warm = binding.PatternDict(ctx, mcfg.n_clusters, mcfg.n_q_heads, mcfg.seq, B)
+                    warm.prefill_attn_layer(Ll["q"], Ll["k"], Ll["v"], Ll["cluster_map"], gamma, 0.3, 0.2, B, mout, stream=stream)
+                    torch.cuda.synchronize()
+                    warm.close()
+                de = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                de[0].record(stream)
+                pd.prefill_attn_layer(Ll["q"], Ll["k"], Ll["v"], Ll["cluster_map"], gamma, 0.3, 0.2, B, mout,
+                                      pattern_out=mpat, stream=stream)
+                de[1].record(stream)
+                torch.cuda.synchronize()
+                t_layers += de[0].elapsed_time(de[1])
+                lp = mpat.cpu().numpy()
+                for c in (0, 1, 2):
+                    totals[c] += int((lp == c).sum())
+                new_pivots.append(pd.count() - before)
+                if layer:
+                    del Ll
+            mixed["layer_stack_with_dictionary"] = {
+                "layers": n_dict_layers, "ms_total": t_layers, "ms_per_layer_mean": t_layers / n_dict_layers,
+                "pivots_per_model": pd.count(), "new_pivots_per_layer": new_pivots,
+                "heads_dense_shared_vslash_total": totals,
+                "note": "layers share the heavy key positions and the cluster table (structure seed) and draw their own "
+                        "q, k, v; one sp_prefill_attn_layer call per layer, CUDA events around each call"}
+            pd.close()
+        assert ctx.status() == (0, 0), "device-side wait timed out"
+        del Lm, mout
+        torch.cuda.empty_cache()
+
     # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
     literal = None
     if rank == 0 and not args.no_literal:
@@ -591,6 +649,7 @@ def run_ours(args):
         "paper_literal_pattern": literal,
         "layer_stack": stack,
         "other_configs": others,
+        "mixed_workload": mixed,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -620,6 +679,8 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-mixed", action="store_true",
+                    help="skip the two-family workload (sp_prefill_attn_auto and the dictionary flow at the paper's thresholds)")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the compact block on the other configurations (gamma 0.8 / 0.95, 32K, 64K GQA-7)")
     ap.add_argument("--stack-layers", type=int, default=None,

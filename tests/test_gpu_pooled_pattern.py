@@ -466,6 +466,81 @@ def test_layers_with_cross_layer_dictionary(binding, pooled):
     assert d.count() == 0
 
 
+# ------------------------------------------------------------------ a workload on which the paper's thresholds decide
+
+def test_mixed_workload_at_the_papers_thresholds(binding):
+    """Two families of heads (flat block-averaged last rows / strong local decay) at gamma 0.9, delta 0.3, tau 0.2
+    (Section 6, Implementation Details): the flat family shares its pivots' patterns, the other one falls back to
+    vertical-slash, in sp_prefill_attn_auto and in the dictionary flow (where only the flat family yields pivots)."""
+    from oracle import shareprefill_oracle as orc
+    cfg = synth.scaled(synth.CONFIGS["llama8b_128k_mixed"], 8192)
+    L = synth.make_layer(cfg, seed=2)
+    B, Nb, Hq = cfg.block, cfg.seq // cfg.block, cfg.n_q_heads
+    G = Hq // cfg.n_kv_heads
+    gamma, delta, tau = 0.9, 0.3, 0.2
+    cm, piv = list(L["cluster_map"]), list(L["pivot_heads"])
+    Q, K, V = par.f64(L["q"]), par.f64(L["k"]), par.f64(L["v"])
+    a_hat = [ppo.last_block_distribution(Q[h], K[h // G], B) for h in range(Hq)]
+    want = {}
+    for h in range(Hq):
+        if h in piv:
+            want[h] = 0
+            continue
+        pat, ds, dm = ppo.determine_pattern(a_hat[h], a_hat[piv[cm[h]]], delta, tau)
+        assert min(abs(ds - delta), abs(dm - tau)) > 0.05          # the families are far from the thresholds
+        want[h] = 1 if pat == "shared_pivot" else 2
+    assert {1, 2} <= set(want.values())
+    ctx = binding.Context()
+    q, k, v = L["q"].cuda(), L["k"].cuda(), L["v"].cuda()
+    tri = np.tril(np.ones((Nb, Nb), np.uint8))
+
+    def check_outputs(out, mask_h, pat_h, label):
+        picks = {}
+        for h in range(Hq):
+            picks.setdefault(int(pat_h[h]), h)
+        assert set(picks) == {0, 1, 2}
+        for code, h in picks.items():
+            M = tri if code == 0 else mask_h[h]
+            par.assert_out_close(par.f64(out[h]), orc.masked_attention(Q, K, V, h, M, B), f"{label} head {h} pattern {code}")
+        assert torch.isfinite(out.float()).all()
+
+    out = torch.full_like(q, float("nan"))
+    mask = torch.full((Hq, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
+    pat = torch.full((Hq,), -1, dtype=torch.int32, device="cuda")
+    ctx.sp_prefill_attn_auto(q, k, v, cm, piv, gamma, delta, tau, B, out, mask_out=mask, pattern_out=pat)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    pat_h, mask_h = pat.cpu().numpy(), mask.cpu().numpy()
+    assert [int(x) for x in pat_h] == [want[h] for h in range(Hq)]
+    for h in range(Hq):
+        if pat_h[h] == 1:
+            assert np.array_equal(mask_h[h], mask_h[piv[cm[h]]])
+    check_outputs(out, mask_h, pat_h, "auto")
+
+    # the dictionary flow decides the pivots itself: a head of the other family never becomes one
+    d = binding.PatternDict(ctx, cfg.n_clusters, Hq, cfg.seq, B)
+    out2 = torch.full_like(q, float("nan"))
+    mask.fill_(7)
+    pat.fill_(-1)
+    d.prefill_attn_layer(q, k, v, cm, gamma, delta, tau, B, out2, mask_out=mask, pattern_out=pat)
+    torch.cuda.synchronize()
+    assert ctx.status() == (0, 0)
+    pat_h, mask_h = pat.cpu().numpy(), mask.cpu().numpy()
+    u = np.full(Nb, 1.0 / Nb)
+    seen = set()
+    for h in range(Hq):
+        sparse = ppo.js_distance(a_hat[h], u) >= delta
+        if sparse:
+            assert pat_h[h] == 2
+        elif cm[h] not in seen:
+            seen.add(cm[h])
+            assert pat_h[h] == 0
+        else:
+            assert pat_h[h] == 1
+    assert d.count() == len(seen) == cfg.global_clusters
+    check_outputs(out2, mask_h, pat_h, "dictionary")
+
+
 # ------------------------------------------------------------------ the same calls at the sizes the benchmark times
 
 def _lines_mask(gv, gs, Nb, B, N):
