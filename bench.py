@@ -307,7 +307,8 @@ def run_ours(args):
 
     cfg = workload_cfg(args)
     gamma = args.gamma
-    L = synth.make_layer(cfg, seed=rank_seed(args.seed, rank), device=str(dev))
+    by_cluster = args.shard == "cluster" and world > 1      # ONE layer split over the ranks (strong scaling)
+    L = synth.make_layer(cfg, seed=args.seed if by_cluster else rank_seed(args.seed, rank), device=str(dev))
     q, k, v = L["q"], L["k"], L["v"]
     cm, piv = L["cluster_map"], L["pivot_heads"]
     Nb, B = cfg.seq // cfg.block, cfg.block
@@ -323,8 +324,35 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- the layer split by cluster: a shard is the pivots of some clusters, their members and the heads that run
+    #      dense; K and V are replicated, every rank writes the output rows of its own heads, nothing is exchanged
+    from paper_2505_19578_b200 import sharding
+    sh_bufs = {}
+
+    def run_shard(sh):
+        n_p = len(sh.pivots)
+        if n_p not in sh_bufs:
+            sh_bufs[n_p] = (torch.empty(max(n_p, 1), Nb, Nb, device=dev),
+                            torch.empty(max(n_p, 1), Nb, Nb, dtype=torch.uint8, device=dev),
+                            torch.empty(max(n_p, 1), Nb, dtype=torch.int32, device=dev),
+                            torch.empty(max(n_p, 1), Nb, Nb, dtype=torch.int32, device=dev))
+        s_imp, s_pm, s_cnt, s_idx = sh_bufs[n_p]
+        if n_p:
+            ctx.sp_dense_pivot_attn(q, k, v, sh.pivots, B, out, importance_out=s_imp[:n_p], stream=stream)
+            ctx.sp_block_mask_from_importance(s_imp[:n_p], gamma, s_pm[:n_p], s_cnt[:n_p], s_idx[:n_p], stream=stream)
+        if sh.dense:
+            ctx.sp_dense_pivot_attn(q, k, v, sh.dense, B, out, stream=stream)
+        if sh.members:
+            ctx.sp_block_sparse_attn(q, k, v, sh.members, sh.member_list, s_cnt[:max(n_p, 1)], s_idx[:max(n_p, 1)], B, out,
+                                     stream=stream)
+
+    my_shard = sharding.deal_clusters(cm, piv, world, Nb)[rank] if by_cluster else None
+
     def step():
-        ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, B, out, mask_out=mask, stream=stream)
+        if by_cluster:
+            run_shard(my_shard)
+        else:
+            ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, B, out, mask_out=mask, stream=stream)
 
     # ---- warm-up, then the timed region: K whole-layer steps, inputs resident in HBM
     for _ in range(args.warmup):
@@ -395,6 +423,27 @@ def run_ours(args):
         torch.cuda.synchronize()
         dense_ms = d0.elapsed_time(d1) / 2
     clocks = sampler.stop() if rank == 0 else None
+
+    # ---- preview of the split by cluster on this one GPU: the shards of a W-rank run one after the other; the longest
+    #      is what the layer would take on W GPUs (no exchange step; an estimate, not a multi-GPU measurement)
+    shard_preview = None
+    if world == 1 and args.shard_preview > 1:
+        shards = sharding.deal_clusters(cm, piv, args.shard_preview, Nb)
+        per = []
+        for sh in shards:
+            run_shard(sh)
+            torch.cuda.synchronize()
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            p0.record(stream)
+            for _ in range(3):
+                run_shard(sh)
+            p1.record(stream)
+            torch.cuda.synchronize()
+            per.append({"heads": sh.heads(), "pivots": sh.pivots, "estimated_tiles": sh.cost, "ms": p0.elapsed_time(p1) / 3})
+        shard_preview = {"ranks": args.shard_preview, "shards": per, "ms_longest": max(x["ms"] for x in per),
+                         "ms_sum": sum(x["ms"] for x in per),
+                         "note": "shards timed one after the other on ONE GPU; ms_longest estimates the layer at that many "
+                                 "GPUs with K/V replicated (no collective in the path)"}
 
     # ---- optional: a stack of layers (each its own seeded inputs and 3-6 clusters), times summed over layers
     stack = None
@@ -592,7 +641,7 @@ def run_ours(args):
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
     d2h = hout.numel() * hout.element_size()
 
-    ms, layers = aggregate(ms_local, 1.0, world, dev)
+    ms, layers = aggregate(ms_local, 1.0 / world if by_cluster else 1.0, world, dev)
     e2e_ms, _ = aggregate(e2e_ms_local, 1.0, world, dev)
     if rank != 0:
         if world > 1:
@@ -624,12 +673,14 @@ def run_ours(args):
     mask_bytes = len(piv) * Nb * Nb * (4 + 1 + 4) + len(piv) * Nb * 4
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if by_cluster else "weak", "vs_baseline": None,
+        "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
                    "head_dim": cfg.head_dim, "block": cfg.block, "gamma": gamma, "n_pivots": len(piv),
                    "seed": args.seed, "l2": "inputs (2.5 GiB at 128K) exceed the 126 MB L2; no flush between steps",
-                   "units_per_rank": "one layer per rank, independent seeds"},
+                   "units_per_rank": ("one layer split by cluster over the ranks (K/V replicated, outputs disjoint, no "
+                                      "collective)" if by_cluster else "one layer per rank, independent seeds")},
         "ms_per_layer": ms,
         "kernels_ms": {"pivot_dense_attn": k1, "block_mask": k2, "block_sparse_attn": k3},
         "visited_tiles": {"pivot": pivot_tiles, "members": member_tiles, "causal_per_head": tiles_causal},
@@ -650,6 +701,7 @@ def run_ours(args):
         "layer_stack": stack,
         "other_configs": others,
         "mixed_workload": mixed,
+        "shard_preview": shard_preview,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -679,6 +731,11 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="override the workload's sequence length (profiling on a small case)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--shard", default="layer", choices=["layer", "cluster"],
+                    help="with --gpus N > 1: 'layer' = one independent layer per rank (weak scaling, default); 'cluster' = ONE "
+                         "layer split by head cluster over the ranks (strong scaling, no collective)")
+    ap.add_argument("--shard-preview", type=int, default=0,
+                    help="at N = 1: also time the shards of a split by cluster over this many ranks, one after the other")
     ap.add_argument("--no-mixed", action="store_true",
                     help="skip the two-family workload (sp_prefill_attn_auto and the dictionary flow at the paper's thresholds)")
     ap.add_argument("--no-other-configs", action="store_true",

@@ -250,7 +250,9 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
  * members run in groups of four heads, each group's outputs copied back while
  * the next group computes.  Copies use two streams owned by the context; when the
  * call returns everything is enqueued, and `stream` is made to wait for the last
- * copy, so synchronising `stream` is enough before reading out_host.
+ * copy, so synchronising `stream` is enough before reading out_host.  The same
+ * holds when the call fails part-way: whatever copies it had already enqueued
+ * are joined into `stream` before it returns the error.
  *
  *   q_host             host bf16 [n_q_heads, seq, head_dim], contiguous
  *   k_host, v_host     host bf16 [n_kv_heads, seq, head_dim], contiguous

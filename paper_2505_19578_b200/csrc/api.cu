@@ -656,23 +656,30 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
     return SP_OK;
   };
 
+  // From here on the copy streams may hold work: on any failure both are joined into the caller's stream before the
+  // call returns, so that synchronising `stream` is enough before the host buffers are freed or reused.
+  auto bail = [&](int code) {
+    hand_over(sout, sc);
+    hand_over(sin, sc);
+    return code;
+  };
   const int n_first = n_pivots > 1 ? n_pivots - 1 : n_pivots;
-  if ((rc = run_pivots(0, n_first))) return rc;
+  if ((rc = run_pivots(0, n_first))) return bail(rc);
   for (int gkv = 0; gkv < n_kv_heads; ++gkv)
-    if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return SP_ERR_CUDA; kv_sent[gkv] = true; }
-  if (!hand_over(sin, sc)) return SP_ERR_CUDA;                                   // members read every KV head
-  if ((rc = run_members(0, n_first, n_first == n_pivots))) return rc;
+    if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return bail(SP_ERR_CUDA); kv_sent[gkv] = true; }
+  if (!hand_over(sin, sc)) return bail(SP_ERR_CUDA);                             // members read every KV head
+  if ((rc = run_members(0, n_first, n_first == n_pivots))) return bail(rc);
   if (n_first < n_pivots) {
-    if ((rc = run_pivots(n_first, n_pivots))) return rc;
-    if ((rc = run_members(n_first, n_pivots, true))) return rc;
+    if ((rc = run_pivots(n_first, n_pivots))) return bail(rc);
+    if ((rc = run_members(n_first, n_pivots, true))) return bail(rc);
   }
   if (mask_out_host) {
     gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, sc>>>(pmask, mask_src, p.Nb, dmask);
-    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return bail(SP_ERR_CUDA);
     ctx->launches += 1;
-    if (!hand_over(sc, sout)) return SP_ERR_CUDA;
+    if (!hand_over(sc, sout)) return bail(SP_ERR_CUDA);
     if (cudaMemcpyAsync(mask_out_host, dmask, (size_t)p.Hq * p.Nb * p.Nb, cudaMemcpyDeviceToHost, sout) != cudaSuccess)
-      return SP_ERR_CUDA;
+      return bail(SP_ERR_CUDA);
   }
   // the caller's stream ends after the last copy out (and after the last copy in)
   if (!hand_over(sout, sc) || !hand_over(sin, sc)) return SP_ERR_CUDA;

@@ -74,3 +74,57 @@ def test_traffic_table_parsing(tmp_path):
     t = bench.load_traffic_table(str(p))
     assert t == {("llama8b_128k", 131072, 0.9, 0, "pivot_dense_attn"): 123456}
     assert bench.load_traffic_table(str(tmp_path / "missing.txt")) == {}
+
+
+def _shard_worker(rank, world, port, q):
+    import os
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import torch
+    import torch.distributed as dist
+    from paper_2505_19578_b200 import sharding, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    cm, piv = synth.make_cluster_map(synth.CONFIGS["llama8b_128k_mixed"], 0)
+    cm[5] = -1                                         # a head without a cluster: a dense unit of its own
+    shards = sharding.deal_clusters(cm, piv, world, 1024)
+    mine = shards[rank]
+    owned = torch.zeros(len(cm), dtype=torch.int32)
+    owned[mine.heads()] = 1
+    dist.all_reduce(owned)                             # how many ranks compute each head
+    costs = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]
+    dist.all_gather(costs, torch.tensor([mine.cost], dtype=torch.float64))
+    q.put((rank, owned.tolist(), [float(c) for c in costs], mine.pivots, mine.members, mine.member_list, mine.dense))
+    dist.destroy_process_group()
+
+
+def test_cluster_sharding_gloo_world2():
+    """Strong-scaling split of one layer by cluster: every head is computed by exactly one rank, a pivot sits with
+    all the members that walk its list, and the estimated loads are balanced."""
+    import multiprocessing as mp
+    from paper_2505_19578_b200 import sharding, synth
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 500
+    ps = [ctx.Process(target=_shard_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in ps:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in ps)
+    for p in ps:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    cm, piv = synth.make_cluster_map(synth.CONFIGS["llama8b_128k_mixed"], 0)
+    cm[5] = -1
+    for rank, owned, costs, pivots, members, member_list, dense in got:
+        assert owned == [1] * len(cm)                                  # exactly once, on every rank's view
+        for h, slot in zip(members, member_list):
+            assert cm[h] == cm[pivots[slot]] and cm[h] >= 0            # a member walks the list of its own cluster's pivot
+        assert all(p in piv for p in pivots)
+        assert max(costs) <= 1.35 * min(costs)                         # 6 clusters + 1 loose head on 2 ranks
+    assert 5 in got[0][6] + got[1][6]
+    # one rank: everything; more ranks than units: some stay empty, nothing is lost
+    one = sharding.deal_clusters(cm, piv, 1, 64)
+    assert one[0].heads() == list(range(len(cm)))
+    many = sharding.deal_clusters(cm, piv, 16, 64)
+    assert sorted(h for s in many for h in s.heads()) == list(range(len(cm)))
+    # a second listed pivot of a cluster runs dense on the rank of its cluster
+    units, loose = sharding.units_of_layer([0, 0, 0, 1], [0, 1])
+    assert units[0]["pivot"] == 0 and units[0]["extra_pivots"] == [1] and units[0]["members"] == [2] and loose == [3]
