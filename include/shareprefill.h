@@ -188,12 +188,14 @@ int sp_fixed_scratch_status(int device, int* code /* host, out */, int* where /*
  *   budget K whose top-K sum reaches gamma, turn the index set into a mask.)
  *   Each row-block i of each of the `n_maps` maps is treated independently over
  *   its causal entries j = 0..i: order by importance descending (equal values:
- *   smaller j first), running sum in that order in float64, K_i = first k whose
- *   sum >= gamma (all i+1 entries if the sum never gets there); the first K_i
- *   entries of the order are selected.
+ *   smaller j first), running sum in that order, K_i = first k whose sum >= gamma
+ *   (all i+1 entries if the sum never gets there); the first K_i entries of the
+ *   order are selected.  The running sum is exact (fixed point in units of 2^-50:
+ *   it equals a float64 running sum unless that sum passes within 1e-12 of gamma).
  *
- *   importance   device fp32 [n_maps, nb, nb]; entries must be finite and >= 0
- *                (anything else is read as 0); entries with j > i are ignored.
+ *   importance   device fp32 [n_maps, nb, nb]; entries are probabilities: finite and
+ *                >= 0 (anything else is read as 0; an entry above 4 counts as 4 in
+ *                the running sum); entries with j > i are ignored.
  *   gamma        > 0.  Compared as the double nearest to this float.
  *   mask_out     device u8  [n_maps, nb, nb]: 1 = compute, 0 = skip (j > i: 0); may be NULL.
  *   counts_out   device i32 [n_maps, nb]: K_i.

@@ -4,144 +4,107 @@
 // budget K whose top-K sum reaches gamma, select those indices.  Applied to each
 // row-block independently over its causal entries.
 //
-// One warp owns one row.  The row's (score, index) pairs are packed into 64-bit
-// keys, sorted with a bitonic network held entirely in registers (in-lane
-// compare-exchanges for short distances, shuffles for long ones), scanned in
-// float64, cut at gamma, and the selected indices are compacted in ascending
-// order through a shared-memory bitmap + popcount prefix.
+// One warp owns one row, its scores in registers (lane l holds entries l, l + 32,
+// ...).  No sort is needed to know WHICH entries the sorted prefix holds: with
+// T the largest score for which the entries >= T sum to at least gamma, the
+// prefix is every entry above T plus the first few entries equal to T in index
+// order (equal scores go to the smaller key-block).  T is found bit by bit on
+// the fp32 bit patterns (31 passes of a compare, an add and a warp reduction per
+// held entry); the sums are exact fixed-point integers in units of 2^-50 (scores
+// are probabilities: every score >= 2^-27 is represented exactly, smaller ones
+// lose less than 2^-50 each; a score above 4 counts as 4), and integer additions
+// commute, so the result does not depend on the order of the additions.  The
+// selected entries are then written in ascending index order with ballots.
+// A full sort of (score, index) keys in registers (a bitonic network of 55
+// stages for 1024 keys) did the same in three times the instructions.
 #include "common.cuh"
 
 namespace sp {
 namespace {
 
 constexpr int kWarpsPerBlock = 4;
-constexpr int kBitmapWords = kMaxNb / 32;
+constexpr unsigned long long kFxCap = 1ull << 52;   // 4.0 in units of 2^-50: 1024 of them still fit in 64 bits
 
-// Sort key: ascending order of the key == descending score, then ascending index.
-// Scores are finite and >= 0, so their bit patterns order like the values.
-__device__ __forceinline__ uint64_t make_key(float v, int idx) {
-  uint32_t bits = (v > 0.f && v <= 3.4028235e38f) ? __float_as_uint(v) : 0u;
-  return ((uint64_t)(~bits) << 32) | (uint32_t)idx;
+// Finite positive scores only; anything else counts as 0.
+__device__ __forceinline__ uint32_t mask_score_bits(float v) { return (v > 0.f && v <= 3.4028235e38f) ? __float_as_uint(v) : 0u; }
+
+// value * 2^50 of a positive finite fp32 bit pattern (bits below 2^-50 dropped, capped at kFxCap): integer shifts only
+__device__ __forceinline__ unsigned long long mask_score_fixed(uint32_t bits) {
+  const int e = (int)(bits >> 23);
+  const unsigned long long m = (unsigned long long)(bits & 0x7FFFFFu) | (e ? 0x800000ull : 0ull);
+  const int sh = (e ? e : 1) - 150 + 50;          // value = m * 2^((e ? e : 1) - 150)
+  if (sh >= 29) return kFxCap;                    // m < 2^24, so m << 29 could pass the cap
+  if (sh >= 0) { const unsigned long long x = m << sh; return x < kFxCap ? x : kFxCap; }
+  return sh > -64 ? m >> (-sh) : 0ull;
 }
-__device__ __forceinline__ float key_score(uint64_t key) { return __uint_as_float(~(uint32_t)(key >> 32)); }
 
-__device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t x, int m) {
-  uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)x, m);
-  uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(x >> 32), m);
-  return ((uint64_t)hi << 32) | lo;
-}
-
-// Bitonic sort of 32*E keys spread over a warp; sorted position p lives in
-// lane p / E, register p % E.
-template <int E>
-__device__ __forceinline__ void warp_bitonic_sort(uint64_t (&key)[E], int lane) {
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
-  for (int k = 2; k <= 32 * E; k <<= 1) {
-#pragma unroll
-    for (int d = k >> 1; d > 0; d >>= 1) {
-      if (d < E) {
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-          if ((e & d) == 0) {
-            const int p = lane * E + e;
-            const bool up = (p & k) == 0;
-            uint64_t a = key[e], b = key[e | d];
-            const bool sw = (a > b) == up;
-            key[e] = sw ? b : a;
-            key[e | d] = sw ? a : b;
-          }
-        }
-      } else {
-        const int lm = d / E;
-        const bool lower = (lane & lm) == 0;
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-          const int p = lane * E + e;
-          const bool up = (p & k) == 0;
-          uint64_t other = shfl_xor_u64(key[e], lm);
-          uint64_t mn = key[e] < other ? key[e] : other;
-          uint64_t mx = key[e] < other ? other : key[e];
-          key[e] = (lower == up) ? mn : mx;
-        }
-      }
-    }
-  }
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
 }
 
 template <int E>
-__device__ void mask_row(const float* __restrict__ row, int n, int nb, double gamma, uint8_t* mask_row_out,
-                         int32_t* count_out, int32_t* idx_row_out, uint32_t* bitmap, int lane) {
-  uint64_t key[E];
+__device__ void mask_row(const float* __restrict__ row, int n, int nb, unsigned long long gamma_fx, uint8_t* mask_row_out,
+                         int32_t* count_out, int32_t* idx_row_out, int lane) {
+  uint32_t bits[E];
+  unsigned long long fx[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) {
-    const int j = e * 32 + lane;             // coalesced load; the sort does not care where a key starts
-    key[e] = j < n ? make_key(row[j], j) : ~0ull;
+    const int j = e * 32 + lane;
+    bits[e] = j < n ? mask_score_bits(row[j]) : 0u;
+    fx[e] = mask_score_fixed(bits[e]);
   }
-  warp_bitonic_sort<E>(key, lane);
-
-  // running sum in sorted order, float64
-  double val[E];
-  double local = 0.0;
+  auto sum_from = [&](uint32_t t) {
+    unsigned long long s = 0;
 #pragma unroll
-  for (int e = 0; e < E; ++e) {
-    val[e] = key[e] != ~0ull ? (double)key_score(key[e]) : 0.0;
-    local += val[e];
-  }
-  double incl = local;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    double t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  double cum = incl - local;
-  int first = -1;
-#pragma unroll
-  for (int e = 0; e < E; ++e) {
-    cum += val[e];
-    if (first < 0 && key[e] != ~0ull && cum >= gamma) first = lane * E + e;
-  }
-  const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
-  int K = n;
-  if (hit) K = __shfl_sync(0xffffffffu, first, __ffs(hit) - 1) + 1;
-
-  // selected set -> bitmap over key-block indices
-  if (lane < kBitmapWords) bitmap[lane] = 0u;
-  __syncwarp();
-#pragma unroll
-  for (int e = 0; e < E; ++e) {
-    const int p = lane * E + e;
-    if (p < K) {
-      const uint32_t j = (uint32_t)key[e];
-      atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+    for (int e = 0; e < E; ++e)
+      if (bits[e] >= t) s += fx[e];
+    return warp_sum_u64(s);
+  };
+  const unsigned long long total = sum_from(1u);
+  const bool all = total < gamma_fx;              // the scores never reach gamma: every causal entry is selected
+  uint32_t T = 0u, k_eq = 0u;
+  if (!all) {
+#pragma unroll 1
+    for (int bit = 30; bit >= 0; --bit) {
+      const uint32_t cand = T | (1u << bit);
+      if (sum_from(cand) >= gamma_fx) T = cand;
     }
+    const unsigned long long above = sum_from(T + 1u);
+    const unsigned long long v_fx = mask_score_fixed(T);
+    const unsigned long long need = gamma_fx > above ? gamma_fx - above : 1ull;
+    const unsigned long long k = v_fx ? (need + v_fx - 1) / v_fx : ~0ull;
+    k_eq = k > 0xffffffffull ? 0xffffffffu : (uint32_t)k;
   }
-  __syncwarp();
-
-  // ascending compaction
-  uint32_t word = lane < kBitmapWords ? bitmap[lane] : 0u;
-  int c = __popc(word), off = c;
+  // selection in ascending index order: everything above T, then copies of T while they are needed
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t seen_eq = 0u;
+  int cnt = 0;
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, off, o);
-    if (lane >= o) off += t;
+  for (int e = 0; e < E; ++e) {
+    const int j = e * 32 + lane;
+    const bool eq = !all && bits[e] == T && j < n;
+    const uint32_t bal_eq = __ballot_sync(0xffffffffu, eq);
+    const bool on = j < n && (all || bits[e] > T || (eq && seen_eq + __popc(bal_eq & lt) < k_eq));
+    seen_eq += __popc(bal_eq);
+    const uint32_t bal = __ballot_sync(0xffffffffu, on);
+    if (on) idx_row_out[cnt + __popc(bal & lt)] = j;
+    cnt += __popc(bal);
+    if (mask_row_out && j < nb) mask_row_out[j] = (uint8_t)(on ? 1 : 0);
   }
-  off -= c;
-  while (word) {
-    const int b = __ffs(word) - 1;
-    idx_row_out[off++] = lane * 32 + b;
-    word &= word - 1;
-  }
-  for (int j = K + lane; j < nb; j += 32) idx_row_out[j] = -1;
-  if (lane == 0) *count_out = K;
+  for (int j = cnt + lane; j < nb; j += 32) idx_row_out[j] = -1;
   if (mask_row_out)
-    for (int j = lane; j < nb; j += 32) mask_row_out[j] = (uint8_t)((bitmap[j >> 5] >> (j & 31)) & 1u);
-  __syncwarp();
+    for (int j = E * 32 + lane; j < nb; j += 32) mask_row_out[j] = 0;
+  if (lane == 0) *count_out = cnt;
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) block_mask_kernel(const MaskArgs a) {
-  __shared__ uint32_t bitmaps[kWarpsPerBlock][kBitmapWords];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long total = (long)a.n_maps * a.nb;
+  // cumulative >= gamma  <=>  fixed-point cumulative >= ceil(gamma * 2^50)
+  const double gs = a.gamma * 1125899906842624.0;
+  const unsigned long long gamma_fx = gs >= 9.0e18 ? ~0ull : (gs <= 1.0 ? 1ull : (unsigned long long)ceil(gs));
   for (long w = (long)blockIdx.x * kWarpsPerBlock + warp; w < total; w += (long)gridDim.x * kWarpsPerBlock) {
     const int i = a.nb - 1 - (int)(w / a.n_maps);   // long rows first
     const int mp = (int)(w % a.n_maps);
@@ -151,13 +114,12 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) block_mask_kernel(const M
     int32_t* cnt = a.counts + (size_t)mp * a.nb + i;
     int32_t* irow = a.indices + rbase;
     const int n = i + 1;
-    uint32_t* bm = bitmaps[warp];
-    if (n <= 32)        mask_row<1>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
-    else if (n <= 64)   mask_row<2>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
-    else if (n <= 128)  mask_row<4>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
-    else if (n <= 256)  mask_row<8>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
-    else if (n <= 512)  mask_row<16>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
-    else                mask_row<32>(row, n, a.nb, a.gamma, mrow, cnt, irow, bm, lane);
+    if (n <= 32)        mask_row<1>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
+    else if (n <= 64)   mask_row<2>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
+    else if (n <= 128)  mask_row<4>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
+    else if (n <= 256)  mask_row<8>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
+    else if (n <= 512)  mask_row<16>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
+    else                mask_row<32>(row, n, a.nb, gamma_fx, mrow, cnt, irow, lane);
   }
 }
 
