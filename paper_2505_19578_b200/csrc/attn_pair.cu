@@ -170,6 +170,31 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 
+// The tile statistics are written once and read once by the same CTA about an item later; with the K/V tiles
+// streaming through L2 they were evicted to DRAM in between (two thirds of K1's DRAM traffic).  Their lines are
+// therefore stored with the evict-last priority and read with evict-first (dead after the read).
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_f32_hint(float* addr, float v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(addr), "f"(v), "l"(policy) : "memory");
+}
+__device__ __forceinline__ float4 ld_f32x4_hint(const float* addr, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(addr), "l"(policy)
+               : "memory");
+  return v;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -598,6 +623,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     const bool tthread = row == 0;
     // per-CTA statistics region: [tile][step of the item][row]
     float* const stats = a.tile_stats ? a.tile_stats + ((size_t)blockIdx.x * 2 + x) * (size_t)a.Nb * BLK : nullptr;
+    const uint64_t pol_keep = l2_policy_evict_last(), pol_done = l2_policy_evict_first();
     int ts = 0;          // steps of this tile so far, over all items (parity of S_FULL and of the P hand-offs)
     int on = 0;          // items in which this tile had work so far (parity of O_DONE)
     bool fail = false;   // a wait of this thread ran out
@@ -721,7 +747,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         if (tthread) trace(trole, 15, t);
         // off the critical path: running sum and the tile statistic
         l += tile_sum;
-        if (emit) stats[(size_t)t * BLK + row] = m_ref + log2f(tile_sum);
+        if (emit) st_f32_hint(stats + (size_t)t * BLK + row, m_ref + log2f(tile_sum), pol_keep);
       }
       if (ok) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_O_DONE + x), (uint32_t)on & 1u, ab, 32 + x));
@@ -769,7 +795,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               const int t = t0 + 4 * e;
-              v[e] = t < cnt ? *reinterpret_cast<const float4*>(stats + (size_t)t * BLK + lane * 4)
+              v[e] = t < cnt ? ld_f32x4_hint(stats + (size_t)t * BLK + lane * 4, pol_done)
                              : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
             }
 #pragma unroll
