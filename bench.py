@@ -553,7 +553,7 @@ def run_ours(args):
     # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
     literal = None
     if rank == 0 and not args.no_literal:
-        pooled = torch.empty(len(piv), Nb, Nb, device=dev)
+        pooled = torch.empty(len(piv), Nb, Nb, dtype=torch.float64, device=dev)
         lm = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device=dev)
         lc = torch.empty(len(piv), Nb, dtype=torch.int32, device=dev)
         li = torch.empty(len(piv), Nb, Nb, dtype=torch.int32, device=dev)

@@ -283,8 +283,10 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
  *   q_r . k_c / sqrt(head_dim) over the visible (c <= r) entries of the block of
  *   head heads[t]; entries with j > i are -infinity.  The mean over a full block
  *   equals the product of the block means of Q and K, which is how it is
- *   computed (fp32).
- *     heads host [n_heads]; pooled_out device fp32 [n_heads, Nb, Nb].
+ *   computed, in float64 (the cut below compares a cumulative sum over up to half a
+ *   million scores with gamma; fp32 averages of logits of order 1..30 would move it
+ *   by 1e-5).
+ *     heads host [n_heads]; pooled_out device FLOAT64 [n_heads, Nb, Nb].
  *
  * sp_pattern_from_pooled - Algorithm "Construct Pivotal Pattern": softmax of the
  *   block averages along each row-block, the last row kept as the pivotal
@@ -292,14 +294,17 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
  *   descending (equal scores: smaller row-major index first), minimum budget K
  *   whose scores sum to >= gamma (every existing block if they never do), index
  *   set -> mask.  A row-block left without a selected block receives its diagonal
- *   block.  Outputs as for sp_block_mask_from_importance (mask_out required),
- *   plus last_row_out device fp32 [n_maps, nb] or NULL.
+ *   block.  The softmax is taken in float64 and every score rounded to fp32 once;
+ *   the cumulative sums are exact fixed-point sums of those fp32 scores.
+ *     pooled device FLOAT64 [n_maps, nb, nb] (as written by sp_pooled_logits).
+ *   Outputs as for sp_block_mask_from_importance (mask_out required), plus
+ *   last_row_out device fp32 [n_maps, nb] or NULL.
  *
  * sp_determine_pattern - Algorithm "Determine Sparse Pattern": a^ = softmax of
  *   the pooled QK values of the last block of queries against every key-block,
  *   d_sparse = sqrt(JSD(a^ || uniform)), d_sim = sqrt(JSD(a^ || a~)) (natural
- *   logarithm), pattern = shared pivot iff d_sparse < delta and d_sim < tau,
- *   else vertical-slash.
+ *   logarithm, float64 arithmetic on the device, the distances returned as fp32),
+ *   pattern = shared pivot iff d_sparse < delta and d_sim < tau, else vertical-slash.
  *     pivot_last_rows device fp32 [n_rows, Nb] (a~ of the pivots, as written by
  *     sp_pattern_from_pooled); row_of_head host [n_heads]: which row each head is
  *     compared with, -1 = none (d_sim = +infinity).
@@ -307,8 +312,8 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
  *     dist_out device fp32 [n_heads, 2] = (d_sparse, d_sim), or NULL.
  */
 int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads,
-                     int n_heads, int block, float* pooled_out, void* stream);
-int sp_pattern_from_pooled(sp_ctx* ctx, const float* pooled, int n_maps, int nb, float gamma,
+                     int n_heads, int block, double* pooled_out, void* stream);
+int sp_pattern_from_pooled(sp_ctx* ctx, const double* pooled, int n_maps, int nb, float gamma,
                            uint8_t* mask_out, int32_t* counts_out, int32_t* indices_out,
                            float* last_row_out, void* stream);
 int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads,

@@ -206,12 +206,13 @@ class Context:
 
     def sp_pooled_logits(self, q, k, heads, block, pooled_out, stream=None):
         heads = list(heads)
+        assert pooled_out.dtype == torch.float64 and pooled_out.is_contiguous(), "the pooled map is float64"
         _check(self._lib.sp_pooled_logits(self._h, _view(q), _view(k), _i32(heads), len(heads), block, _ptr(pooled_out),
                                           _stream(stream)), "sp_pooled_logits")
 
     def sp_pattern_from_pooled(self, pooled, gamma, mask_out, counts_out, indices_out, last_row_out=None, stream=None):
         n_maps, nb, nb2 = pooled.shape
-        assert nb == nb2 and pooled.dtype == torch.float32 and pooled.is_contiguous()
+        assert nb == nb2 and pooled.dtype == torch.float64 and pooled.is_contiguous(), "the pooled map is float64"
         _check(self._lib.sp_pattern_from_pooled(self._h, _ptr(pooled), n_maps, nb, gamma, _ptr(mask_out), _ptr(counts_out),
                                                 _ptr(indices_out), _ptr(last_row_out), _stream(stream)),
                "sp_pattern_from_pooled")

@@ -697,13 +697,13 @@ PooledArgs pooled_args(const Problem& p, const sp_tensor* q, const sp_tensor* k,
   a.k_sh = k->stride[1]; a.k_sn = k->stride[2];
   a.group = p.Hq / p.Hkv; a.B = p.B; a.Nb = p.Nb; a.d = p.d; a.n_heads = n_heads;
   for (int t = 0; t < n_heads; ++t) a.heads.v[t] = heads[t];
-  a.scale = (float)(1.0 / sqrt((double)p.d));
+  a.scale = 1.0 / sqrt((double)p.d);
   return a;
 }
 }  // namespace
 
 int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const int32_t* heads, int n_heads, int block,
-                     float* pooled_out, void* stream) {
+                     double* pooled_out, void* stream) {
   if (!ctx || !heads || n_heads < 0 || !pooled_out) return SP_ERR_INVALID_ARG;
   Problem p;
   int rc = check_problem(q, k, k, q, block, &p);
@@ -714,9 +714,9 @@ int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const 
   if (n_heads == 0) return SP_OK;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SP_ERR_CUDA;
-  if ((rc = reserve(ctx, align_up(pooled_scratch_floats(n_heads, p.Nb, p.d) * sizeof(float))))) return rc;
+  if ((rc = reserve(ctx, align_up(pooled_scratch_bytes(n_heads, p.Nb, p.d))))) return rc;
   PooledArgs a = pooled_args(p, q, k, heads, n_heads);
-  a.qbar = static_cast<float*>(ctx->ws);
+  a.qbar = static_cast<double*>(ctx->ws);
   a.kbar = a.qbar + (size_t)n_heads * p.Nb * p.d;
   a.diag = a.kbar + (size_t)n_heads * p.Nb * p.d;
   a.pooled = pooled_out;
@@ -725,7 +725,7 @@ int sp_pooled_logits(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const 
   return SP_OK;
 }
 
-int sp_pattern_from_pooled(sp_ctx* ctx, const float* pooled, int n_maps, int nb, float gamma, uint8_t* mask_out,
+int sp_pattern_from_pooled(sp_ctx* ctx, const double* pooled, int n_maps, int nb, float gamma, uint8_t* mask_out,
                            int32_t* counts_out, int32_t* indices_out, float* last_row_out, void* stream) {
   if (!ctx || !pooled || !mask_out || !counts_out || !indices_out || n_maps < 0 || nb <= 0) return SP_ERR_INVALID_ARG;
   if (!(gamma > 0.f)) return SP_ERR_INVALID_ARG;
@@ -759,9 +759,9 @@ int sp_determine_pattern(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   if (n_heads == 0) return SP_OK;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SP_ERR_CUDA;
-  if ((rc = reserve(ctx, align_up((size_t)n_heads * p.Nb * sizeof(float))))) return rc;
+  if ((rc = reserve(ctx, align_up((size_t)n_heads * p.Nb * sizeof(double))))) return rc;
   PooledArgs a = pooled_args(p, q, k, heads, n_heads);
-  a.pooled = static_cast<float*>(ctx->ws);
+  a.pooled = static_cast<double*>(ctx->ws);
   if (launch_determine_pattern(a, pivot_last_rows, rows, delta, tau, pattern_out, dist_out,
                                static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return SP_ERR_CUDA;
@@ -849,15 +849,15 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   const int n_row = n_pivots > n_members ? n_pivots : n_members;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
-  const size_t o_imp = take(n_pivots * nn * sizeof(float));
+  const size_t o_imp = take(n_pivots * nn * (pooled_construction ? sizeof(double) : sizeof(float)));   // importance, or the pooled map
   const size_t o_scores = take(pooled_construction ? n_pivots * nn * sizeof(float) : 0);
   const size_t o_mask = take(n_lists * nn);
   const size_t o_counts = take((size_t)n_lists * p.Nb * sizeof(int32_t));
   const size_t o_indices = take(n_lists * nn * sizeof(int32_t));
-  const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_pivots, p.Nb, p.d) * sizeof(float)
+  const size_t o_scratch = take(pooled_construction ? pooled_scratch_bytes(n_pivots, p.Nb, p.d)
                                                     : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_pivots, p.Nb, p.B));
   const size_t o_atilde = take((size_t)n_pivots * p.Nb * sizeof(float));
-  const size_t o_rows = take((size_t)n_row * p.Nb * sizeof(float));
+  const size_t o_rows = take((size_t)n_row * p.Nb * sizeof(double));
   const size_t o_small = take((size_t)(3 * kMaxHeads + p.Hq) * sizeof(int32_t));
   const size_t o_vs = take(vslash_scratch_bytes(n_members, p.N, 8));
   if ((rc = reserve(ctx, off))) return rc;
@@ -867,7 +867,7 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   int32_t* counts = reinterpret_cast<int32_t*>(ws + o_counts);
   int32_t* indices = reinterpret_cast<int32_t*>(ws + o_indices);
   float* a_tilde = reinterpret_cast<float*>(ws + o_atilde);
-  float* rows_scratch = reinterpret_cast<float*>(ws + o_rows);
+  double* rows_scratch = reinterpret_cast<double*>(ws + o_rows);
   int32_t* decide = reinterpret_cast<int32_t*>(ws + o_small);
   int32_t* lists_dev = decide + kMaxHeads;
   int32_t* active = lists_dev + kMaxHeads;
@@ -887,12 +887,12 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   if (n_pivots > 0) {
     if (pooled_construction) {
       PooledArgs pa = pooled_args(p, q, k, pivot_heads, n_pivots);
-      pa.qbar = reinterpret_cast<float*>(ws + o_scratch);
+      pa.qbar = reinterpret_cast<double*>(ws + o_scratch);
       pa.kbar = pa.qbar + (size_t)n_pivots * p.Nb * p.d;
       pa.diag = pa.kbar + (size_t)n_pivots * p.Nb * p.d;
-      pa.pooled = imp;
+      pa.pooled = reinterpret_cast<double*>(imp);
       if (launch_pooled_logits(pa, s) != cudaSuccess) return SP_ERR_CUDA;
-      if (launch_pattern_from_pooled(imp, n_pivots, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores), masks, counts,
+      if (launch_pattern_from_pooled(reinterpret_cast<const double*>(imp), n_pivots, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores), masks, counts,
                                      indices, nullptr, s) != cudaSuccess)
         return SP_ERR_CUDA;
       ctx->launches += 5;
@@ -1032,17 +1032,17 @@ int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   const size_t o_ahat = take((size_t)p.Hq * p.Nb * sizeof(float));
-  const size_t o_rows = take((size_t)p.Hq * p.Nb * sizeof(float));
+  const size_t o_rows = take((size_t)p.Hq * p.Nb * sizeof(double));
   const size_t o_small = take((size_t)(4 * kMaxHeads) * sizeof(int32_t) + (size_t)kMaxHeads * sizeof(float));
-  const size_t o_imp = take(n_new_max * nn * sizeof(float));
+  const size_t o_imp = take(n_new_max * nn * (pooled_construction ? sizeof(double) : sizeof(float)));
   const size_t o_scores = take(pooled_construction ? nn * sizeof(float) : 0);
-  const size_t o_scratch = take(pooled_construction ? pooled_scratch_floats(n_new_max, p.Nb, p.d) * sizeof(float)
+  const size_t o_scratch = take(pooled_construction ? pooled_scratch_bytes(n_new_max, p.Nb, p.d)
                                                     : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_new_max, p.Nb, p.B));
   const size_t o_vs = take(vslash_scratch_bytes(p.Hq, p.N, 8));
   if ((rc = reserve(ctx, off))) return rc;
   char* ws = static_cast<char*>(ctx->ws);
   float* a_hat = reinterpret_cast<float*>(ws + o_ahat);
-  float* rows_scratch = reinterpret_cast<float*>(ws + o_rows);
+  double* rows_scratch = reinterpret_cast<double*>(ws + o_rows);
   int32_t* decide = reinterpret_cast<int32_t*>(ws + o_small);
   int32_t* lists_dev = decide + kMaxHeads;
   int32_t* active = lists_dev + kMaxHeads;
@@ -1112,17 +1112,17 @@ int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q
       int ph[kMaxHeads];
       for (int t = 0; t < n_piv; ++t) ph[t] = piv_heads.v[t];
       PooledArgs pp = pooled_args(p, q, k, ph, n_piv);
-      pp.qbar = reinterpret_cast<float*>(ws + o_scratch);
+      pp.qbar = reinterpret_cast<double*>(ws + o_scratch);
       pp.kbar = pp.qbar + (size_t)n_piv * p.Nb * p.d;
       pp.diag = pp.kbar + (size_t)n_piv * p.Nb * p.d;
-      pp.pooled = imp;
+      pp.pooled = reinterpret_cast<double*>(imp);
       if (launch_pooled_logits(pp, s) != cudaSuccess) return SP_ERR_CUDA;
       ctx->launches += 2;
     }
     for (int t = 0; t < n_piv; ++t) {
       const int c = piv_slots.v[t];
       if (pooled_construction) {
-        if (launch_pattern_from_pooled(imp + (size_t)t * nn, 1, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores),
+        if (launch_pattern_from_pooled(reinterpret_cast<const double*>(imp) + (size_t)t * nn, 1, p.Nb, (double)gamma, reinterpret_cast<float*>(ws + o_scores),
                                        dict->masks + (size_t)c * nn, dict->counts + (size_t)c * p.Nb,
                                        dict->indices + (size_t)c * nn, nullptr, s) != cudaSuccess)
           return SP_ERR_CUDA;

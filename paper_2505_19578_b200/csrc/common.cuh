@@ -65,11 +65,11 @@ struct PooledArgs {
   int64_t q_sh, q_sn, k_sh, k_sn;
   int group, B, Nb, d, n_heads;
   HeadTable heads;
-  float scale;     // 1 / sqrt(d)
-  float* qbar;     // scratch [n_heads, Nb, d]: block means of Q
-  float* kbar;     // scratch [n_heads, Nb, d]: block means of K (of the head's KV head)
-  float* diag;     // scratch [n_heads, Nb]: average of the diagonal block's visible entries, scaled
-  float* pooled;   // out [n_heads, Nb, Nb]  (launch_determine_pattern: [n_heads, Nb], the last row only)
+  double scale;    // 1 / sqrt(d)
+  double* qbar;    // scratch [n_heads, Nb, d]: block means of Q
+  double* kbar;    // scratch [n_heads, Nb, d]: block means of K (of the head's KV head)
+  double* diag;    // scratch [n_heads, Nb]: average of the diagonal block's visible entries, scaled
+  double* pooled;  // out [n_heads, Nb, Nb]  (launch_determine_pattern: [n_heads, Nb], the last row only)
 };
 
 // Vertical-slash search (Algorithm "Search Vertical Slash Pattern").  Strides in elements.
@@ -108,9 +108,9 @@ cudaError_t fixed_status_read(int device, int* code, int* where);
 constexpr size_t kFixedScratchBytes = 64ull << 20;
 cudaError_t launch_block_mask(const MaskArgs& a, cudaStream_t s);
 cudaError_t launch_fill_causal_mask(uint8_t* mask, int nb, cudaStream_t s);
-size_t pooled_scratch_floats(int n_heads, int Nb, int d);
+size_t pooled_scratch_bytes(int n_heads, int Nb, int d);
 cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s);
-cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
+cudaError_t launch_pattern_from_pooled(const double* pooled, int n_maps, int nb, double gamma, float* scores,
                                        uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
                                        cudaStream_t s);
 cudaError_t launch_js_uniform(const float* dist, int n, int nb, float* d_sparse, cudaStream_t s);

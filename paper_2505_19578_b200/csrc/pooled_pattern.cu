@@ -36,32 +36,45 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
+// The block means, their products, the softmax over them and the divergences are carried in float64: the
+// global cut compares a cumulative sum of a million scores with gamma, and fp32 means and logits (of order 1..30)
+// would move that sum by 1e-5; with float64 up to the scores (rounded to fp32 once) it moves by under 1e-7.
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_max(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
 
 // ---- block means of Q and K, and the average of the diagonal block ------------------------
 // grid (Nb, n_heads), d threads: thread = one head-dim column.
 __global__ void block_means_kernel(const PooledArgs a) {
-  __shared__ float red[4];
+  __shared__ double red[4];
   const int i = blockIdx.x, slot = blockIdx.y, col = threadIdx.x;
   const int h = a.heads.v[slot], g = h / a.group;
   const __nv_bfloat16* q = a.q + (size_t)h * a.q_sh + (size_t)i * a.B * a.q_sn + col;
   const __nv_bfloat16* k = a.k + (size_t)g * a.k_sh + (size_t)i * a.B * a.k_sn + col;
-  float qsum = 0.f, kcum = 0.f, acc = 0.f;
+  double qsum = 0.0, kcum = 0.0, acc = 0.0;
   for (int r = 0; r < a.B; ++r) {
-    const float qv = __bfloat162float(q[(size_t)r * a.q_sn]);
-    kcum += __bfloat162float(k[(size_t)r * a.k_sn]);
+    const double qv = (double)__bfloat162float(q[(size_t)r * a.q_sn]);
+    kcum += (double)__bfloat162float(k[(size_t)r * a.k_sn]);
     qsum += qv;
-    acc = fmaf(qv, kcum, acc);          // q_r . (k_0 + ... + k_r): the visible half of the diagonal block
+    acc = fma(qv, kcum, acc);           // q_r . (k_0 + ... + k_r): the visible half of the diagonal block
   }
-  const float inv = 1.f / (float)a.B;
+  const double inv = 1.0 / (double)a.B;
   a.qbar[((size_t)slot * a.Nb + i) * a.d + col] = qsum * inv;
   a.kbar[((size_t)slot * a.Nb + i) * a.d + col] = kcum * inv;
   acc = warp_sum(acc);
   if ((col & 31) == 0) red[col >> 5] = acc;
   __syncthreads();
   if (col == 0) {
-    float t = 0.f;
+    double t = 0.0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-    a.diag[(size_t)slot * a.Nb + i] = t * a.scale / (0.5f * (float)a.B * (float)(a.B + 1));
+    a.diag[(size_t)slot * a.Nb + i] = t * a.scale / (0.5 * (double)a.B * (double)(a.B + 1));
   }
 }
 
@@ -70,40 +83,40 @@ __global__ void block_means_kernel(const PooledArgs a) {
 __global__ void pooled_logits_kernel(const PooledArgs a) {
   const int i = blockIdx.x, slot = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float* qb = a.qbar + ((size_t)slot * a.Nb + i) * a.d;
-  float* out = a.pooled + ((size_t)slot * a.Nb + i) * a.Nb;
+  const double* qb = a.qbar + ((size_t)slot * a.Nb + i) * a.d;
+  double* out = a.pooled + ((size_t)slot * a.Nb + i) * a.Nb;
   const int per = a.d / 32;              // 2 or 4 consecutive columns per lane
-  float qv[4];
+  double qv[4];
   for (int e = 0; e < per; ++e) qv[e] = qb[lane * per + e];
   for (int j = warp; j < i; j += 4) {
-    const float* kb = a.kbar + ((size_t)slot * a.Nb + j) * a.d;
-    float acc = 0.f;
-    for (int e = 0; e < per; ++e) acc = fmaf(qv[e], kb[lane * per + e], acc);
+    const double* kb = a.kbar + ((size_t)slot * a.Nb + j) * a.d;
+    double acc = 0.0;
+    for (int e = 0; e < per; ++e) acc = fma(qv[e], kb[lane * per + e], acc);
     acc = warp_sum(acc);
     if (lane == 0) out[j] = acc * a.scale;
   }
   if (threadIdx.x == 0) out[i] = a.diag[(size_t)slot * a.Nb + i];
-  for (int j = i + 1 + (int)threadIdx.x; j < a.Nb; j += blockDim.x) out[j] = -CUDART_INF_F;
+  for (int j = i + 1 + (int)threadIdx.x; j < a.Nb; j += blockDim.x) out[j] = -CUDART_INF;
 }
 
 // ---- row-wise softmax of the block averages; one warp per row -------------------------------
-__global__ void pooled_softmax_kernel(const float* __restrict__ pooled, int n_maps, int nb, float* __restrict__ scores,
+__global__ void pooled_softmax_kernel(const double* __restrict__ pooled, int n_maps, int nb, float* __restrict__ scores,
                                       float* __restrict__ last_row) {
   const int lane = threadIdx.x & 31;
   const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (w >= (long)n_maps * nb) return;
   const int mp = (int)(w / nb), i = (int)(w % nb);
-  const float* row = pooled + ((size_t)mp * nb + i) * nb;
+  const double* row = pooled + ((size_t)mp * nb + i) * nb;
   float* out = scores + ((size_t)mp * nb + i) * nb;
-  float m = -CUDART_INF_F;
-  for (int j = lane; j <= i; j += 32) m = fmaxf(m, row[j]);
+  double m = -CUDART_INF;
+  for (int j = lane; j <= i; j += 32) m = fmax(m, row[j]);
   m = warp_max(m);
-  float s = 0.f;
-  for (int j = lane; j <= i; j += 32) s += expf(row[j] - m);
+  double s = 0.0;
+  for (int j = lane; j <= i; j += 32) s += exp(row[j] - m);
   s = warp_sum(s);
-  const float inv = 1.f / s;
+  const double inv = 1.0 / s;
   for (int j = lane; j < nb; j += 32) {
-    const float p = j <= i ? expf(row[j] - m) * inv : 0.f;
+    const float p = j <= i ? (float)(exp(row[j] - m) * inv) : 0.f;      // the one rounding to fp32
     out[j] = p;
     if (last_row && i == nb - 1) last_row[(size_t)mp * nb + j] = p;
   }
@@ -223,87 +236,87 @@ __global__ void compact_rows_kernel(uint8_t* __restrict__ mask, int n_maps, int 
 // pooled last row: grid (Nb, n_heads), d threads.  Block j: mean of the last query block against the mean
 // of key block j; the last block uses the visible half.
 __global__ void last_row_pooled_kernel(const PooledArgs a) {
-  __shared__ float red[4];
+  __shared__ double red[4];
   const int j = blockIdx.x, slot = blockIdx.y, col = threadIdx.x;
   const int h = a.heads.v[slot], g = h / a.group;
   const int last = a.Nb - 1;
   const __nv_bfloat16* q = a.q + (size_t)h * a.q_sh + (size_t)last * a.B * a.q_sn + col;
   const __nv_bfloat16* k = a.k + (size_t)g * a.k_sh + (size_t)j * a.B * a.k_sn + col;
-  float acc = 0.f, denom;
+  double acc = 0.0, denom;
   if (j < last) {
-    float qsum = 0.f, ksum = 0.f;
+    double qsum = 0.0, ksum = 0.0;
     for (int r = 0; r < a.B; ++r) {
-      qsum += __bfloat162float(q[(size_t)r * a.q_sn]);
-      ksum += __bfloat162float(k[(size_t)r * a.k_sn]);
+      qsum += (double)__bfloat162float(q[(size_t)r * a.q_sn]);
+      ksum += (double)__bfloat162float(k[(size_t)r * a.k_sn]);
     }
     acc = qsum * ksum;
-    denom = (float)a.B * (float)a.B;
+    denom = (double)a.B * (double)a.B;
   } else {
-    float kcum = 0.f;
+    double kcum = 0.0;
     for (int r = 0; r < a.B; ++r) {
-      kcum += __bfloat162float(k[(size_t)r * a.k_sn]);
-      acc = fmaf(__bfloat162float(q[(size_t)r * a.q_sn]), kcum, acc);
+      kcum += (double)__bfloat162float(k[(size_t)r * a.k_sn]);
+      acc = fma((double)__bfloat162float(q[(size_t)r * a.q_sn]), kcum, acc);
     }
-    denom = 0.5f * (float)a.B * (float)(a.B + 1);
+    denom = 0.5 * (double)a.B * (double)(a.B + 1);
   }
   acc = warp_sum(acc);
   if ((col & 31) == 0) red[col >> 5] = acc;
   __syncthreads();
   if (col == 0) {
-    float t = 0.f;
+    double t = 0.0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
     a.pooled[(size_t)slot * a.Nb + j] = t * a.scale / denom;
   }
 }
 
 // one CTA of 256 threads per head: softmax of the pooled last row, the two Jensen-Shannon distances, the decision
-__global__ void decide_pattern_kernel(const float* __restrict__ pooled_last, int nb, const float* __restrict__ pivot_rows,
+__global__ void decide_pattern_kernel(const double* __restrict__ pooled_last, int nb, const float* __restrict__ pivot_rows,
                                       HeadTable row_of_head, float delta, float tau, int32_t* __restrict__ pattern,
                                       float* __restrict__ dist) {
-  __shared__ float red[8];
-  __shared__ float bc[2];
+  __shared__ double red[8];
+  __shared__ double bc[2];
   const int slot = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* z = pooled_last + (size_t)slot * nb;
+  const double* z = pooled_last + (size_t)slot * nb;
   const int prow = row_of_head.v[slot];
   const float* at = prow >= 0 ? pivot_rows + (size_t)prow * nb : nullptr;
-  auto block_reduce = [&](float v, bool is_max) {
+  auto block_reduce = [&](double v, bool is_max) {
     v = is_max ? warp_max(v) : warp_sum(v);
     __syncthreads();
     if (lane == 0) red[warp] = v;
     __syncthreads();
     if (tid == 0) {
-      float t = red[0];
-      for (int w = 1; w < (int)(blockDim.x >> 5); ++w) t = is_max ? fmaxf(t, red[w]) : t + red[w];
+      double t = red[0];
+      for (int w = 1; w < (int)(blockDim.x >> 5); ++w) t = is_max ? fmax(t, red[w]) : t + red[w];
       bc[0] = t;
     }
     __syncthreads();
     return bc[0];
   };
-  float m = -CUDART_INF_F;
-  for (int j = tid; j < nb; j += blockDim.x) m = fmaxf(m, z[j]);
+  double m = -CUDART_INF;
+  for (int j = tid; j < nb; j += blockDim.x) m = fmax(m, z[j]);
   m = block_reduce(m, true);
-  float s = 0.f;
-  for (int j = tid; j < nb; j += blockDim.x) s += expf(z[j] - m);
+  double s = 0.0;
+  for (int j = tid; j < nb; j += blockDim.x) s += exp(z[j] - m);
   s = block_reduce(s, false);
-  const float inv = 1.f / s, u = 1.f / (float)nb;
+  const double inv = 1.0 / s, u = 1.0 / (double)nb;
   // JSD(p || q) = 1/2 sum p ln(p/m) + 1/2 sum q ln(q/m), m = (p + q)/2, 0 ln 0 = 0
-  float js_u = 0.f, js_a = 0.f;
+  double js_u = 0.0, js_a = 0.0;
   for (int j = tid; j < nb; j += blockDim.x) {
-    const float p = expf(z[j] - m) * inv;
+    const double p = exp(z[j] - m) * inv;
     {
-      const float mm = 0.5f * (p + u);
-      js_u += (p > 0.f ? p * logf(p / mm) : 0.f) + u * logf(u / mm);
+      const double mm = 0.5 * (p + u);
+      js_u += (p > 0.0 ? p * log(p / mm) : 0.0) + u * log(u / mm);
     }
     if (at) {
-      const float q = at[j], mm = 0.5f * (p + q);
-      js_a += (p > 0.f ? p * logf(p / mm) : 0.f) + (q > 0.f ? q * logf(q / mm) : 0.f);
+      const double q = (double)at[j], mm = 0.5 * (p + q);
+      js_a += (p > 0.0 ? p * log(p / mm) : 0.0) + (q > 0.0 ? q * log(q / mm) : 0.0);
     }
   }
   js_u = block_reduce(js_u, false);
   js_a = block_reduce(js_a, false);
   if (tid == 0) {
-    const float d_sparse = sqrtf(fmaxf(0.5f * js_u, 0.f));
-    const float d_sim = at ? sqrtf(fmaxf(0.5f * js_a, 0.f)) : CUDART_INF_F;
+    const float d_sparse = (float)sqrt(fmax(0.5 * js_u, 0.0));
+    const float d_sim = at ? (float)sqrt(fmax(0.5 * js_a, 0.0)) : CUDART_INF_F;
     pattern[slot] = (d_sparse < delta && d_sim < tau) ? 0 : 1;
     if (dist) { dist[2 * slot] = d_sparse; dist[2 * slot + 1] = d_sim; }
   }
@@ -311,7 +324,7 @@ __global__ void decide_pattern_kernel(const float* __restrict__ pooled_last, int
 
 }  // namespace
 
-size_t pooled_scratch_floats(int n_heads, int Nb, int d) { return (size_t)n_heads * Nb * (2 * (size_t)d + 1); }
+size_t pooled_scratch_bytes(int n_heads, int Nb, int d) { return (size_t)n_heads * Nb * (2 * (size_t)d + 1) * sizeof(double); }
 
 cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s) {
   if (a.n_heads == 0) return cudaSuccess;
@@ -320,7 +333,7 @@ cudaError_t launch_pooled_logits(const PooledArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, double gamma, float* scores,
+cudaError_t launch_pattern_from_pooled(const double* pooled, int n_maps, int nb, double gamma, float* scores,
                                        uint8_t* mask, int32_t* counts, int32_t* indices, float* last_row,
                                        cudaStream_t s) {
   if (n_maps == 0) return cudaSuccess;
@@ -334,29 +347,29 @@ cudaError_t launch_pattern_from_pooled(const float* pooled, int n_maps, int nb, 
 namespace {
 
 // softmax of each row of z [n, nb] -> out; one CTA of 256 threads per row
-__global__ void row_softmax_kernel(const float* __restrict__ z, int nb, float* __restrict__ out) {
-  __shared__ float red[8];
-  __shared__ float bc;
+__global__ void row_softmax_kernel(const double* __restrict__ z, int nb, float* __restrict__ out) {
+  __shared__ double red[8];
+  __shared__ double bc;
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* in = z + (size_t)row * nb;
-  float m = -CUDART_INF_F;
-  for (int j = tid; j < nb; j += blockDim.x) m = fmaxf(m, in[j]);
+  const double* in = z + (size_t)row * nb;
+  double m = -CUDART_INF;
+  for (int j = tid; j < nb; j += blockDim.x) m = fmax(m, in[j]);
   m = warp_max(m);
   if (lane == 0) red[warp] = m;
   __syncthreads();
-  if (tid == 0) { float t = red[0]; for (int w = 1; w < 8; ++w) t = fmaxf(t, red[w]); bc = t; }
+  if (tid == 0) { double t = red[0]; for (int w = 1; w < 8; ++w) t = fmax(t, red[w]); bc = t; }
   __syncthreads();
   m = bc;
-  float s = 0.f;
-  for (int j = tid; j < nb; j += blockDim.x) s += expf(in[j] - m);
+  double s = 0.0;
+  for (int j = tid; j < nb; j += blockDim.x) s += exp(in[j] - m);
   s = warp_sum(s);
   __syncthreads();
   if (lane == 0) red[warp] = s;
   __syncthreads();
-  if (tid == 0) { float t = 0.f; for (int w = 0; w < 8; ++w) t += red[w]; bc = t; }
+  if (tid == 0) { double t = 0.0; for (int w = 0; w < 8; ++w) t += red[w]; bc = t; }
   __syncthreads();
-  const float inv = 1.f / bc;
-  for (int j = tid; j < nb; j += blockDim.x) out[(size_t)row * nb + j] = expf(in[j] - m) * inv;
+  const double inv = 1.0 / bc;
+  for (int j = tid; j < nb; j += blockDim.x) out[(size_t)row * nb + j] = (float)(exp(in[j] - m) * inv);
 }
 
 }  // namespace
@@ -397,22 +410,22 @@ __global__ void finalize_pattern_kernel(const int32_t* __restrict__ decide, Head
 namespace {
 // sqrt(JSD(a^ || uniform)) of each row of dist [n, nb]; one CTA of 256 threads per row
 __global__ void js_uniform_kernel(const float* __restrict__ dist, int nb, float* __restrict__ d_sparse) {
-  __shared__ float red[8];
+  __shared__ double red[8];
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* p_ = dist + (size_t)row * nb;
-  const float u = 1.f / (float)nb;
-  float js = 0.f;
+  const double u = 1.0 / (double)nb;
+  double js = 0.0;
   for (int j = tid; j < nb; j += blockDim.x) {
-    const float p = p_[j], mm = 0.5f * (p + u);
-    js += (p > 0.f ? p * logf(p / mm) : 0.f) + u * logf(u / mm);
+    const double p = (double)p_[j], mm = 0.5 * (p + u);
+    js += (p > 0.0 ? p * log(p / mm) : 0.0) + u * log(u / mm);
   }
   js = warp_sum(js);
   if (lane == 0) red[warp] = js;
   __syncthreads();
   if (tid == 0) {
-    float t = 0.f;
+    double t = 0.0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-    d_sparse[row] = sqrtf(fmaxf(0.5f * t, 0.f));
+    d_sparse[row] = (float)sqrt(fmax(0.5 * t, 0.0));
   }
 }
 
@@ -420,24 +433,24 @@ __global__ void js_uniform_kernel(const float* __restrict__ dist, int nb, float*
 // a_hat [Hq, nb] indexed by head, a_tilde [n_slots, nb]; one CTA of 256 threads per listed head.
 __global__ void js_pair_decide_kernel(const float* __restrict__ a_hat, const float* __restrict__ a_tilde, int nb,
                                       HeadTable heads, HeadTable slot_of, float tau, int32_t* __restrict__ decide) {
-  __shared__ float red[8];
+  __shared__ double red[8];
   const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sl = slot_of.v[t];
   if (sl < 0) { if (tid == 0) decide[t] = 1; return; }
   const float* p_ = a_hat + (size_t)heads.v[t] * nb;
   const float* q_ = a_tilde + (size_t)sl * nb;
-  float js = 0.f;
+  double js = 0.0;
   for (int j = tid; j < nb; j += blockDim.x) {
-    const float p = p_[j], q = q_[j], mm = 0.5f * (p + q);
-    js += (p > 0.f ? p * logf(p / mm) : 0.f) + (q > 0.f ? q * logf(q / mm) : 0.f);
+    const double p = (double)p_[j], q = (double)q_[j], mm = 0.5 * (p + q);
+    js += (p > 0.0 ? p * log(p / mm) : 0.0) + (q > 0.0 ? q * log(q / mm) : 0.0);
   }
   js = warp_sum(js);
   if (lane == 0) red[warp] = js;
   __syncthreads();
   if (tid == 0) {
-    float s = 0.f;
+    double s = 0.0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
-    decide[t] = sqrtf(fmaxf(0.5f * s, 0.f)) < tau ? 0 : 1;
+    decide[t] = (float)sqrt(fmax(0.5 * s, 0.0)) < tau ? 0 : 1;
   }
 }
 

@@ -10,11 +10,12 @@ from tests import _parity as par
 
 pytestmark = pytest.mark.gpu
 
-POOLED_ATOL = 2e-5     # fp32 block means and dot products of bf16 data, logits of order 1..30
-SCORE_BAND = 2e-5      # an entry may flip only if the oracle's cumulative score at it is this close to gamma
-DIV_ATOL = 2e-6        # Jensen-Shannon divergences (squared distances) from fp32 distributions;
-                       # the square root amplifies rounding near zero, so the squares are compared
-DIST_MARGIN = 2e-3     # a decision is checked when both distances are this far from their thresholds
+POOLED_ATOL = 1e-10    # float64 block means and dot products of bf16 data on both sides (other summation order)
+SCORE_BAND = 1e-6      # an entry may flip only if the oracle's cumulative score at it is this close to gamma: the
+                       # library's scores are float64 softmax values rounded to fp32 once (6e-8 relative), summed exactly
+DIV_ATOL = 1e-7        # Jensen-Shannon divergences (squared distances): float64 arithmetic on a representative that is
+                       # stored in fp32 (6e-8 relative); the squares are compared (the root amplifies rounding near 0)
+DIST_MARGIN = 1e-4     # a decision is checked when both distances are this far from their thresholds
 
 
 @pytest.fixture(scope="module")
@@ -73,7 +74,7 @@ def test_pooled_logits_and_pattern_match_oracle(binding, name, seq, gamma):
     heads = list(L["pivot_heads"]) + [h for h in range(cfg.n_q_heads) if h not in L["pivot_heads"]][:1]
     ctx = binding.Context()
     q, k = L["q"].cuda(), L["k"].cuda()
-    pooled = torch.full((len(heads), Nb, Nb), float("nan"), device="cuda")
+    pooled = torch.full((len(heads), Nb, Nb), float("nan"), dtype=torch.float64, device="cuda")
     ctx.sp_pooled_logits(q, k, heads, B, pooled)
     mask = torch.full((len(heads), Nb, Nb), 7, dtype=torch.uint8, device="cuda")
     counts = torch.full((len(heads), Nb), -5, dtype=torch.int32, device="cuda")
@@ -109,7 +110,7 @@ def test_pattern_from_pooled_exact_cases(binding):
     # equal scores inside a row (ties go to the smaller index), forced diagonals, unreachable gamma; the
     # gammas stay clear of the cumulative sums 1/8, 3/16, 1/4, ... where fp32 scores could fall either way
     Nb = 8
-    At = np.where(np.tril(np.ones((Nb, Nb), bool)), 0.0, -np.inf).astype(np.float32)     # uniform rows: scores 1/(i+1)
+    At = np.where(np.tril(np.ones((Nb, Nb), bool)), 0.0, -np.inf)                        # uniform rows: scores 1/(i+1)
     ctx = binding.Context()
     pooled = torch.from_numpy(np.stack([At, At])).cuda()
     for gamma in (0.15, 0.2, 0.26, 0.6, 0.9, 1e-6, 1.5):
@@ -118,7 +119,7 @@ def test_pattern_from_pooled_exact_cases(binding):
         idx = torch.zeros(2, Nb, Nb, dtype=torch.int32, device="cuda")
         ctx.sp_pattern_from_pooled(pooled, gamma, mask, counts, idx)
         torch.cuda.synchronize()
-        res = ppo.construct_pivotal_pattern(At.astype(np.float64), par.gamma32(gamma))
+        res = ppo.construct_pivotal_pattern(At, par.gamma32(gamma))
         for t in range(2):
             assert np.array_equal(mask[t].cpu().numpy(), res["mask"]), gamma
             assert np.array_equal(counts[t].cpu().numpy(), res["mask"].sum(axis=1))
@@ -132,7 +133,7 @@ def test_determine_pattern_matches_oracle(binding, name, seq):
     piv = list(L["pivot_heads"])
     ctx = binding.Context()
     q, k = L["q"].cuda(), L["k"].cuda()
-    pooled = torch.empty(len(piv), Nb, Nb, device="cuda")
+    pooled = torch.empty(len(piv), Nb, Nb, dtype=torch.float64, device="cuda")
     ctx.sp_pooled_logits(q, k, piv, B, pooled)
     mask = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device="cuda")
     counts = torch.empty(len(piv), Nb, dtype=torch.int32, device="cuda")
@@ -177,12 +178,14 @@ def test_determine_pattern_matches_oracle(binding, name, seq):
     # a pivot compared with its own representative: distance 0
     for t, p in enumerate(piv):
         if rows[p] == t:
-            assert got_d[p, 1] <= 2e-3
+            assert got_d[p, 1] <= 5e-4
 
 
 # ------------------------------------------------------------------ vertical-slash search
 
-VS_BAND = 2e-5         # a line may flip only if the oracle's cumulative score at it is this close to gamma
+VS_BAND = 2e-5         # a line may flip only if the oracle's cumulative score at it is this close to gamma: the
+                       # probabilities come from bf16 tensor-core products accumulated in fp32 (128 terms of size up to
+                       # ~2, logits up to ~30 after scaling: about 2e-5 absolute on a logit, i.e. relative on a score)
 
 
 def _cum_at(a, g):
@@ -308,7 +311,7 @@ def test_prefill_attn_auto_is_the_composition_of_its_steps(binding, name, seq, p
 
     # masks: pivots' as the construction call gives them, members' by their decision
     if pooled:
-        pl = torch.empty(len(piv), Nb, Nb, device="cuda")
+        pl = torch.empty(len(piv), Nb, Nb, dtype=torch.float64, device="cuda")
         ctx.sp_pooled_logits(q, k, piv, B, pl)
         pmask = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device="cuda")
         pc = torch.empty(len(piv), Nb, dtype=torch.int32, device="cuda")
@@ -667,7 +670,7 @@ def test_pooled_construction_at_full_size(binding, name, gamma):
     G = cfg.n_q_heads // cfg.n_kv_heads
     h = L["pivot_heads"][0]
     ctx = binding.Context()
-    pooled = torch.full((1, Nb, Nb), float("nan"), device="cuda")
+    pooled = torch.full((1, Nb, Nb), float("nan"), dtype=torch.float64, device="cuda")
     ctx.sp_pooled_logits(L["q"], L["k"], [h], B, pooled)
     torch.cuda.synchronize()
     At = ppo.pooled_logits(par.f64(L["q"][h].cpu()), par.f64(L["k"][h // G].cpu()), B)
@@ -679,7 +682,7 @@ def test_pooled_construction_at_full_size(binding, name, gamma):
     g = par.gamma32(gamma)
     res, cum_at, flat = _oracle_cut(At, g)
     n_diff = {}
-    for label, src in (("own map", pooled), ("oracle's map", torch.from_numpy(At[None].astype(np.float32)).cuda())):
+    for label, src in (("own map", pooled), ("oracle's map", torch.from_numpy(At[None].copy()).cuda())):
         mask = torch.full((1, Nb, Nb), 7, dtype=torch.uint8, device="cuda")
         counts = torch.full((1, Nb), -5, dtype=torch.int32, device="cuda")
         idx = torch.full((1, Nb, Nb), -5, dtype=torch.int32, device="cuda")
@@ -704,7 +707,7 @@ def test_invalid_arguments_of_the_pattern_calls(binding):
     k = torch.zeros(2, 512, 128, dtype=torch.bfloat16, device="cuda")
     out = torch.zeros_like(q)
     Nb = 4
-    f = torch.zeros(1, Nb, Nb, device="cuda")
+    f = torch.zeros(1, Nb, Nb, dtype=torch.float64, device="cuda")
     m = torch.zeros(1, Nb, Nb, dtype=torch.uint8, device="cuda")
     c = torch.zeros(1, Nb, dtype=torch.int32, device="cuda")
     ix = torch.zeros(1, Nb, Nb, dtype=torch.int32, device="cuda")
