@@ -59,7 +59,8 @@ enum {
   SP_ERR_WORKSPACE = -3,   /* workspace allocation failed                              */
   SP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                      */
   SP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (see sp_get_status)   */
-  SP_ERR_SCRATCH_LIMIT = -6 /* sp_dense_pivot_attn_fixed_scratch: problem too large for the fixed array */
+  SP_ERR_SCRATCH_LIMIT = -6, /* sp_dense_pivot_attn_fixed_scratch: problem too large for the fixed array */
+  SP_ERR_RANGE = -7         /* range-checked debug build only: an index left its range (see sp_get_status) */
 };
 
 /* bf16 tensor view: device pointer, sizes and strides in ELEMENTS. */
@@ -96,7 +97,12 @@ int sp_ctx_reserve(sp_ctx* ctx, size_t bytes);
 
 /* Read and clear the device status word.  The caller must have synchronised
  * the stream(s) it used.  *code is SP_OK or SP_ERR_TIMEOUT; *where identifies
- * the wait that gave up (kernel-internal id).  Either pointer may be NULL. */
+ * the wait that gave up (kernel-internal id).  Either pointer may be NULL.
+ * The range-checked debug build of the library (compiled with SP_DEBUG; the
+ * stand-in for a memory checker) also reports SP_ERR_RANGE here: an index that a
+ * kernel computed from its inputs (a listed key-block, a head, a statistics
+ * slot) was out of range; the kernel then used the nearest valid index instead
+ * of touching memory it does not own, and *where names the check. */
 int sp_get_status(sp_ctx* ctx, int* code /* host, out */, int* where /* host, out */);
 
 /* Self-test of the bounded device-side waits: launches one warp that waits,

@@ -14,7 +14,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libshareprefill.so")
+# SHAREPREFILL_LIB: load this library instead of the in-tree release build (e.g. the range-checked debug build,
+# paper_2505_19578_b200/libshareprefill_debug.so, made by `python -m paper_2505_19578_b200.build --debug`)
+LIB_PATH = os.environ.get("SHAREPREFILL_LIB") or os.path.join(_HERE, "libshareprefill.so")
 
 SP_OK = 0
 SP_ERR_INVALID_ARG = -1
@@ -23,6 +25,7 @@ SP_ERR_WORKSPACE = -3
 SP_ERR_CUDA = -4
 SP_ERR_TIMEOUT = -5
 SP_ERR_SCRATCH_LIMIT = -6
+SP_ERR_RANGE = -7
 FIXED_SCRATCH_BYTES = 64 << 20
 
 EXPORTS = (

@@ -203,6 +203,7 @@ const char* sp_strerror(int code) {
     case SP_ERR_CUDA: return "CUDA call failed";
     case SP_ERR_TIMEOUT: return "device-side wait timed out";
     case SP_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's fixed scratch array holds";
+    case SP_ERR_RANGE: return "an index left its range (range-checked debug build)";
     default: return "unknown error code";
   }
 }

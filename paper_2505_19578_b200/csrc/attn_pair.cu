@@ -362,7 +362,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
               it.id = raw;
               it.slot = a.order.v[a.group_start.v[g] + rest % ng];
               it.u = n_pairs - 1 - rest / ng;
-              it.h = a.heads.v[it.slot];
+              it.slot = sp_in_range(it.slot, 0, a.n_heads - 1, a.status, 51);
+              it.h = sp_in_range(a.heads.v[it.slot], 0, a.n_q_heads - 1, a.status, 51);
               it.list = a.lists_dev ? a.lists_dev[it.slot] : a.lists.v[it.slot];
               if (it.list < 0) it.list = -1;
               int cnt[2];
@@ -422,13 +423,15 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         while ((pa < cntA || pb < cntB) && ok) {
           const int ja = pa < cntA ? (listed ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
           const int jb = pb < cntB ? (listed ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
-          const int j = ja < jb ? ja : jb;
-          int f = (ja == j ? F_A : 0) | (jb == j ? F_B : 0);
-          if (ja == j) {
+          const int j_listed = ja < jb ? ja : jb;
+          int f = (ja == j_listed ? F_A : 0) | (jb == j_listed ? F_B : 0);
+          // a listed key-block lies on or before the diagonal of the later tile that walks it
+          const int j = sp_in_range(j_listed, 0, (f & F_B) ? iB : iA, a.status, 50);
+          if (ja == j_listed) {
             ++pa;
             if (listed && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
           }
-          if (jb == j) {
+          if (jb == j_listed) {
             ++pb;
             if (listed && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
           }
@@ -747,7 +750,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         if (tthread) trace(trole, 15, t);
         // off the critical path: running sum and the tile statistic
         l += tile_sum;
-        if (emit) st_f32_hint(stats + (size_t)t * BLK + row, m_ref + log2f(tile_sum), pol_keep);
+        if (emit) st_f32_hint(stats + (size_t)sp_in_range(t, 0, a.Nb - 1, a.status, 52) * BLK + row, m_ref + log2f(tile_sum), pol_keep);
       }
       if (ok) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_O_DONE + x), (uint32_t)on & 1u, ab, 32 + x));

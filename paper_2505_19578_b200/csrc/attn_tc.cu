@@ -134,7 +134,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
       int issued_k = 0, issued_v = 0;
       bool ok = true;
       for (int t = 0; t < cnt && ok; ++t) {
-        const int j = idx ? idx[t] : t;
+        const int j = sp_in_range(idx ? idx[t] : t, 0, i, a.status, 60);
         if (t > 0) ok = mbar_wait(bar(BAR_QK_DONE), (t - 1) & 1, ab, 10);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_K_FULL), P::KV_TX);
@@ -208,7 +208,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
     float m_ref = -CUDART_INF_F, l = 0.f;
     bool ok = cnt > 0;
     for (int t = 0; t < cnt && ok; ++t) {
-      const int j = idx ? idx[t] : t;
+      const int j = sp_in_range(idx ? idx[t] : t, 0, i, a.status, 60);
       ok = mbar_wait(bar(BAR_QK_DONE), t & 1, ab, 30);
       if (!ok) break;
       tc_fence_after();
@@ -245,7 +245,7 @@ attn_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, const
       }
       l = l * alpha + sum;
       if (threadIdx.x == 0) trace(2, 13, t);
-      if (emit && row_valid) stats[(size_t)t * BLK + row] = m_new + log2f(sum);
+      if (emit && row_valid) stats[(size_t)sp_in_range(t, 0, i, a.status, 61) * BLK + row] = m_new + log2f(sum);
       if (t > 0 && __any_sync(0xffffffffu, m_new != m_ref)) {
         // O of the previous steps is relative to the old reference: bring it to the new one
 #pragma unroll

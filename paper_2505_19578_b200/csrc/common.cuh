@@ -13,6 +13,21 @@ namespace sp {
 constexpr int kMaxHeads = 128;   // query heads per call (kernel-parameter tables)
 constexpr int kMaxNb = 1024;     // key-blocks per row (mask kernel sorts one row per warp)
 
+// Range checks of the debug build (-DSP_DEBUG): sp_in_range(v, lo, hi, status, where) returns v when lo <= v <= hi;
+// otherwise it records (SP_ERR_RANGE, where) in the status word (first failure wins) and returns the nearest bound,
+// so that the access that follows stays inside memory the kernel owns.  The release build compiles it to `v`.
+// `where` ids: 50 listed key-block (paired kernel), 51 head / slot of a work item, 52 statistics step,
+// 60 listed key-block (one-row-block kernel), 61 its statistics step.
+#ifdef SP_DEBUG
+__device__ __forceinline__ int sp_in_range(int v, int lo, int hi, int* status, int where) {
+  if (v >= lo && v <= hi) return v;
+  if (atomicCAS(status, 0, (int)SP_ERR_RANGE) == 0) status[1] = where;
+  return v < lo ? lo : hi;
+}
+#else
+__device__ __forceinline__ int sp_in_range(int v, int, int, int*, int) { return v; }
+#endif
+
 struct HeadTable {
   int32_t v[kMaxHeads];
 };
