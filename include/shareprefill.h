@@ -98,6 +98,9 @@ int sp_ctx_reserve(sp_ctx* ctx, size_t bytes);
 /* Read and clear the device status word.  The caller must have synchronised
  * the stream(s) it used.  *code is SP_OK or SP_ERR_TIMEOUT; *where identifies
  * the wait that gave up (kernel-internal id).  Either pointer may be NULL.
+ * SP_ERR_UNSUPPORTED with *where = 90 means the device laid out a CTA's shared
+ * memory window or tensor memory differently from what the attention kernel was
+ * built for (it then does no work).
  * The range-checked debug build of the library (compiled with SP_DEBUG; the
  * stand-in for a memory checker) also reports SP_ERR_RANGE here: an index that a
  * kernel computed from its inputs (a listed key-block, a head, a statistics

@@ -45,18 +45,32 @@
 // tiles then fall into step, their softmax phases coincide and nothing overlaps
 // the MMAs.)  P (bf16) overwrites the first half of the S columns it came from
 // and is the TMEM A operand of PV; the next QK of that tile is issued after the
-// PV that reads P, and the tensor pipe keeps issue order.  The softmax finds the
-// row max of the whole tile first, so that P can be handed over in two halves:
-// the PV of keys 0..63 runs while keys 64..127 are still being exponentiated.
+// PV that reads P, and the tensor pipe keeps issue order.
+//
+// What bounds the kernel is the issuing warp.  The tensor pipe accepts an MMA
+// only a couple of instructions ahead, and the issuing thread needs about twenty
+// dependent instructions per tcgen05.mma (election, moves into uniform
+// registers), on a scheduler it shares with two softmax warps: with the softmax
+// arithmetic switched off (timing-only copy) a key-block still took 3200 cycles
+// against 2048 of tensor work, 3750 with it.  So everything the issuing warp
+// does per key-block is kept short: every shared-memory descriptor and barrier
+// address is a compile-time constant (dynamic shared memory starts at offset
+// 0x400 of the CTA's window and a whole-TMEM allocation at column 0; both are
+// checked at kernel start, and the loop is unrolled over the two ring stages so
+// that the stage is a constant too), and P is handed over once per tile and
+// key-block (handing it over in two halves let the first PV start earlier but
+// cost the issuing warp two more barrier syncs per key-block: 2 % slower).
 //
 // Hand-offs.  Completion of MMAs and of TMA copies arrives on mbarriers
 // (tcgen05.commit, complete_tx).  What the issuing warp waits for comes through
 // named barriers instead: a poll of an mbarrier is a shared-memory round trip,
 // 150-250 cycles while the tensor pipe streams operands at the shared-memory
-// limit, and the issuing warp needs five or more hand-offs per key-block.  The
-// softmax warps `bar.arrive` when a half of P is stored, the producer warp
-// relays "K of the next key-block and V of this one have landed", the issuing
-// warp `bar.sync`s.
+// limit (probing them one key-block ahead was tried: 1 % slower than the relay).
+// The softmax warps `bar.arrive` when P is stored, the producer warp relays "K
+// of the next key-block and V of this one have landed", the issuing warp
+// `bar.sync`s.  The relay ids are taken in turn over four barriers: the producer
+// makes the last relay of an item right after the one before it, so two arrivals
+// can be pending before the issuing warp has taken the first.
 //
 // Block importance in one pass: as in the single-tile kernel, each softmax
 // thread spills one float per visited tile, stat = m + log2(sum_c 2^(s_c - m))
@@ -74,6 +88,8 @@
 // step it was in, on ids taken in turn so that an early arrival never lands in
 // a phase the issuing warp has not left; the issuing warp looks at the abort
 // flag after the last sync of every key-block).
+#include <type_traits>
+
 #include "tc_ptx.cuh"
 
 namespace sp {
@@ -121,8 +137,9 @@ enum { F_A = 1, F_B = 2, F_LAST = 4 };
 // Named barriers (0 is __syncthreads, 1 and 2 the epilogues of the two tiles): P of tile x ready (the four softmax
 // warps of the tile arrive, the issuing warp syncs), and K/V tiles of a merged key-block landed (the producer warp
 // arrives, the issuing warp syncs).  Ids are taken in turn — two per tile for P, four for K/V — so that an arrival
-// that comes early, e.g. the release after a wait ran out, never lands in a phase the other side has not left yet.
-enum { NB_P = 3, NB_KV = 11 };   // P: id NB_P + 4 * tile + 2 * half + (step & 1); K/V: id NB_KV + (key-block & 3)
+// that comes early (the producer's last relay of an item, the release after a wait ran out) never lands in a phase
+// the other side has not left yet.
+enum { NB_P = 3, NB_KV = 11 };   // P: id NB_P + 4 * tile + 2 + (step & 1); K/V: id NB_KV + (relay & 3)
 
 // ------------------------------------------------------------------ small PTX helpers of this kernel
 
@@ -205,6 +222,37 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
+}
+
+
+// Compile-time shared-memory addresses: dynamic shared memory starts at this offset of the CTA's shared window
+// (checked at kernel start), so every descriptor and barrier address of the issuing warp is a constant.
+constexpr uint32_t kSmemBase = 0x400;
+constexpr uint64_t desc_c(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+constexpr uint32_t bar_c(int which) { return kSmemBase + kMiscOff + 8u * (uint32_t)which; }
+template <int X, int ST>
+__device__ __forceinline__ void issue_qk_c() {     // S_X = Q_X K^T from K stage ST
+  constexpr uint64_t dq = desc_c(kSmemBase + kQOff + X * kBox, 16, 1024);
+  constexpr uint64_t dk = desc_c(kSmemBase + kKOff + ST * kTile, 16, 1024);
+  constexpr uint32_t idesc = instr_desc(128, BLK, 0, 0);
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) {
+    const uint32_t qoff = ((kk >> 2) * kTile + (kk & 3) * 32) >> 4;
+    const uint32_t koff = ((kk >> 2) * kBox + (kk & 3) * 32) >> 4;
+    mma_ss(kSCol + X * 128, dq + qoff, dk + koff, idesc, kk > 0);
+  }
+  mma_commit(bar_c(BAR_S_FULL + X));
+}
+template <int X, int ST>
+__device__ __forceinline__ void issue_pv_c(bool accumulate) {   // O_X (+)= P_X V from V stage ST
+  constexpr uint64_t dv = desc_c(kSmemBase + kVOff + ST * kTile, kBox, 1024);
+  constexpr uint32_t idesc = instr_desc(128, D, 0, 1);
+#pragma unroll
+  for (int kk = 0; kk < BLK / 16; ++kk)
+    mma_ts(kOCol + X * 128, kSCol + X * 128 + kk * 8, dv + (uint32_t)((kk * 16 * 128) >> 4), idesc, (accumulate || kk > 0) ? 1u : 0u);
 }
 
 // One work item as the scheduler warp posts it to the other roles (shared memory, two slots of eight ints).
@@ -312,6 +360,8 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const bool layout_ok = smem_u32(smem) == kSmemBase && tmem == 0u;
+  if (!layout_ok && threadIdx.x == 0) { if (atomicCAS(a.status, 0, (int)SP_ERR_UNSUPPORTED) == 0) a.status[1] = 90; }
 
   // The k-th item of this CTA, taken by a whole warp.  False when the wait ran out or another role gave up.
   auto take_item = [&](int k, Item& it, int where) -> bool {
@@ -333,7 +383,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
     if (warp == 9) {
       // ---------------------------------------------------------- producer
       const int n_items = a.n_heads * n_pairs;
-      const bool poisoned = *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
+      const bool poisoned = !layout_ok || *reinterpret_cast<volatile int*>(a.status) != 0;   // an earlier wait ran out: do no work
       int gk = 0;        // merged key-blocks of the finished items (ring position of the next item's first)
       int issued_k = 0, issued_v = 0;   // K and V loads issued so far
       int relays = 0;    // relays to the issuing warp so far
@@ -494,32 +544,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       }
     } else if (warp == 8) {
       // ---------------------------------------------------------- MMA issuer
-      constexpr uint32_t idesc_qk = instr_desc(128, BLK, 0, 0);
-      constexpr uint32_t idesc_pv = instr_desc(128, D, 0, 1);
-      // Descriptors differ from these bases only in the 16-byte-unit address field (low word).
-      const uint64_t dq0 = smem_desc(sQ, 16, 1024);
-      const uint64_t dk0 = smem_desc(sK, 16, 1024);
-      const uint64_t dv0 = smem_desc(sV, kBox, 1024);
-      auto issue_qk = [&](int x, int st) {     // S_x = Q_x K^T from K stage st
-        const uint64_t dq = dq0 + (uint64_t)((x * kBox) >> 4);
-        const uint64_t dk = dk0 + (uint64_t)((st * kTile) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t qoff = ((kk >> 2) * kTile + (kk & 3) * 32) >> 4;
-          const uint32_t koff = ((kk >> 2) * kBox + (kk & 3) * 32) >> 4;
-          mma_ss(tmem + kSCol + x * 128, dq + qoff, dk + koff, idesc_qk, kk > 0);
-        }
-        mma_commit(bar(BAR_S_FULL + x));
-      };
-      auto issue_pv = [&](int x, int st, int hf, bool accumulate) {   // O_x (+)= P_x V, keys 64 hf .. 64 hf + 63 of V stage st
-        const uint64_t dv = dv0 + (uint64_t)((st * kTile) >> 4);
-#pragma unroll
-        for (int k4 = 0; k4 < BLK / 32; ++k4) {
-          const int kk = hf * (BLK / 32) + k4;
-          mma_ts(tmem + kOCol + x * 128, tmem + kSCol + x * 128 + kk * 8, dv + (uint32_t)((kk * 16 * 128) >> 4), idesc_pv,
-                 (accumulate || kk > 0) ? 1u : 0u);
-        }
-      };
       int gk = 0;            // merged key-blocks so far, over all items (ring position)
       int relays = 0;        // relays taken from the producer warp so far
       int tA = 0, tB = 0;    // steps of each tile so far, over all items (parity of its P hand-offs)
@@ -540,8 +564,13 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         int f = kflags[gk % kStages];
         if (lane == 0) {
           trace(1, 1, gk);
-          if (f & F_A) issue_qk(0, gk % kStages);
-          if (f & F_B) issue_qk(1, gk % kStages);
+          if (gk & 1) {
+            if (f & F_A) issue_qk_c<0, 1>();
+            if (f & F_B) issue_qk_c<1, 1>();
+          } else {
+            if (f & F_A) issue_qk_c<0, 0>();
+            if (f & F_B) issue_qk_c<1, 0>();
+          }
           mma_commit(bar(BAR_K_EMPTY + gk % kStages));
           if (f & F_LAST) mma_commit(bar(BAR_Q_EMPTY));
           trace(1, 2, gk);
@@ -555,63 +584,54 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         // The first PV of an item overwrites O of the item before: the softmax warps of the tile have read that O
         // out of TMEM before they produced the P this PV waits for.
         int tAl = 0, tBl = 0;  // steps of each tile inside this item
-        for (;;) {
+        auto body = [&](auto st_c) -> bool {       // one merged key-block read from ring stage ST; true: leave the loop
+          constexpr int ST = decltype(st_c)::value, STN = ST ^ 1;
           const bool last = (f & F_LAST) != 0;
-          const int st = gk % kStages, stn = (gk + 1) % kStages;
           bar_sync(NB_KV + (relays & 3), 64);
           ++relays;
-          const int fn_early = last ? 0 : kflags[stn];
-          if (f & F_A) {
-            bar_sync(NB_P + 0 + (tA & 1), 160);
-            tc_fence_after();
-            if (lane == 0) {
-              trace(1, 3, gk);
-              issue_pv(0, st, 0, tAl > 0);
-            }
-            __syncwarp();
-            bar_sync(NB_P + 2 + (tA & 1), 160);
-          }
+          const int fn_early = last ? 0 : kflags[STN];
+          if (f & F_A) bar_sync(NB_P + 2 + (tA & 1), 160);
           tc_fence_after();
           const int fn = fn_early;
           if (lane == 0) {
             if (f & F_A) {
-              issue_pv(0, st, 1, true);
-              if (tAl + 1 == cntA) mma_commit(bar(BAR_O_DONE + 0));
+              trace(1, 3, gk);
+              issue_pv_c<0, ST>(tAl > 0);
+              if (tAl + 1 == cntA) mma_commit(bar_c(BAR_O_DONE + 0));
             }
-            if (fn & F_A) issue_qk(0, stn);
+            if (fn & F_A) issue_qk_c<0, STN>();
             trace(1, 5, gk);
           }
           __syncwarp();
           if (f & F_A) { ++tA; ++tAl; }
-          if (f & F_B) {
-            bar_sync(NB_P + 4 + (tB & 1), 160);
-            tc_fence_after();
-            if (lane == 0) {
-              trace(1, 6, gk);
-              issue_pv(1, st, 0, tBl > 0);
-            }
-            __syncwarp();
-            bar_sync(NB_P + 6 + (tB & 1), 160);
-          }
+          if (f & F_B) bar_sync(NB_P + 6 + (tB & 1), 160);
           const int abort_raw = *abort_flag;       // after all syncs of this key-block; looked at after the MMAs below
           tc_fence_after();
           if (lane == 0) {
             if (f & F_B) {
-              issue_pv(1, st, 1, true);
-              if (tBl + 1 == cntB) mma_commit(bar(BAR_O_DONE + 1));
+              trace(1, 6, gk);
+              issue_pv_c<1, ST>(tBl > 0);
+              if (tBl + 1 == cntB) mma_commit(bar_c(BAR_O_DONE + 1));
             }
-            mma_commit(bar(BAR_V_EMPTY + st));
-            if (fn & F_B) issue_qk(1, stn);
-            if (!last) mma_commit(bar(BAR_K_EMPTY + stn));
-            if (fn & F_LAST) mma_commit(bar(BAR_Q_EMPTY));   // Q of this item has been read for the last time
+            mma_commit(bar_c(BAR_V_EMPTY + ST));
+            if (fn & F_B) issue_qk_c<1, STN>();
+            if (!last) mma_commit(bar_c(BAR_K_EMPTY + STN));
+            if (fn & F_LAST) mma_commit(bar_c(BAR_Q_EMPTY));   // Q of this item has been read for the last time
             trace(1, 4, gk);
           }
           __syncwarp();
           if (f & F_B) { ++tB; ++tBl; }
           ++gk;
           if (__any_sync(0xffffffffu, abort_raw != 0)) ok = false;
-          if (last || !ok) break;
+          if (last || !ok) return true;
           f = fn;
+          return false;
+        };
+        bool done = false;
+        if (gk & 1) done = body(std::integral_constant<int, 1>{});
+        while (!done) {
+          done = body(std::integral_constant<int, 0>{});
+          if (!done) done = body(std::integral_constant<int, 1>{});
         }
       }
     }
@@ -653,8 +673,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + x), (uint32_t)ts & 1u, ab, 30 + x));
         if (!ok) {
           fail = true;
-          bar_arrive(NB_P + 4 * x + 0 + (ts & 1), 160);   // the issuing warp may be at this step's barriers: do not leave it there
-          bar_arrive(NB_P + 4 * x + 2 + (ts & 1), 160);
+          bar_arrive(NB_P + 4 * x + 2 + (ts & 1), 160);   // the issuing warp may be at this step's barrier: do not leave it there
           break;
         }
         tc_fence_after();
@@ -738,9 +757,6 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         reg_fence32(sb);
         mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
         move_reference(mx23, 2);
-        tmem_wait_st();
-        tc_fence_before();
-        bar_arrive(NB_P + 4 * x + 0 + (ts & 1), 160);
         if (tthread) trace(trole, 13, t);
         chunk_exps(sa, 2);
         chunk_exps(sb, 3);
