@@ -678,12 +678,10 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         }
         tc_fence_after();
         if (tthread) trace(trole, 10, t);
-        // The 128 columns are taken as four chunks of 32 (`tcgen05.ld.32x32b.x32`, the next chunk's load in flight).
-        // Chunks 0 and 1 are online-softmax steps of their own: chunk max, (rarely: only when the row max has grown
-        // by more than 2^8) a move of the reference, exponentials, P chunk into columns the sweep has given up.
-        // Then the max of chunks 2 and 3 is taken, and a move they ask for is made, BEFORE the first half of P is
-        // handed over: after that no reference can move in this key-block, so the PV of keys 0..63 may run while
-        // keys 64..127 are exponentiated from the registers they already sit in.
+        // The 128 columns are taken as four chunks of 32 (`tcgen05.ld.32x32b.x32`, the next chunk's load in flight),
+        // each an online-softmax step of its own: chunk max, (rarely: only when the row max has grown by more than
+        // 2^8) a move of the reference, exponentials, P chunk into columns the sweep has given up.  P is handed to
+        // the issuing warp once, after the fourth chunk.
         float tile_sum = 0.f;
         uint32_t sa[32], sb[32];
         if (j == i) mask_diag_tmem(tS, row);
@@ -752,13 +750,12 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
         tmem_ld_wait();
         reg_fence32(sa);
         tmem_ld32_async(tS + 96, sb);
-        float mx23 = chunk_max(sa);
+        move_reference(chunk_max(sa) * scale, 2);
+        chunk_exps(sa, 2);
         tmem_ld_wait();
         reg_fence32(sb);
-        mx23 = fmaxf(mx23, chunk_max(sb)) * scale;
-        move_reference(mx23, 2);
         if (tthread) trace(trole, 13, t);
-        chunk_exps(sa, 2);
+        move_reference(chunk_max(sb) * scale, 3);
         chunk_exps(sb, 3);
         tmem_wait_st();
         tc_fence_before();
