@@ -92,6 +92,14 @@ int sp_ctx_destroy(sp_ctx* ctx);
 int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block,
                        int n_pivots, size_t* bytes /* host, out */);
 
+/* The same for the calls that decide the pattern on the device (head_dim 128, block 128): *auto_bytes for
+ * sp_prefill_attn_auto with n_pivots listed pivots, *layer_bytes for sp_prefill_attn_layer in a layer that
+ * creates at most n_pivots new pivots.  Either pointer may be NULL.  (sp_prefill_attn_host also keeps device
+ * copies of q, k, v and out, 2 q + 2 k sizes, allocated on its first call.) */
+int sp_workspace_bytes_patterns(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block,
+                                int n_pivots, int pooled_construction, size_t* auto_bytes /* host, out */,
+                                size_t* layer_bytes /* host, out */);
+
 /* Make sure the context's workspace holds at least `bytes`. */
 int sp_ctx_reserve(sp_ctx* ctx, size_t bytes);
 

@@ -35,7 +35,7 @@ EXPORTS = (
     "sp_ctx_set_trace", "sp_prefill_attn_host", "sp_pooled_logits", "sp_pattern_from_pooled",
     "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
     "sp_dict_create", "sp_dict_destroy", "sp_dict_clear", "sp_dict_count", "sp_prefill_attn_layer",
-    "sp_selftest_wait_timeout", "sp_fixed_scratch_status",
+    "sp_selftest_wait_timeout", "sp_fixed_scratch_status", "sp_workspace_bytes_patterns",
 )
 
 
@@ -68,6 +68,8 @@ def load() -> ctypes.CDLL:
     lib.sp_ctx_create.argtypes = [ctypes.POINTER(P), I]
     lib.sp_ctx_destroy.argtypes = [P]
     lib.sp_workspace_bytes.argtypes = [ctypes.c_int64, I, I, I, I, I, ctypes.POINTER(ctypes.c_size_t)]
+    lib.sp_workspace_bytes_patterns.argtypes = [ctypes.c_int64, I, I, I, I, I, I, ctypes.POINTER(ctypes.c_size_t),
+                                                ctypes.POINTER(ctypes.c_size_t)]
     lib.sp_ctx_reserve.argtypes = [P, ctypes.c_size_t]
     lib.sp_get_status.argtypes = [P, ctypes.POINTER(I), ctypes.POINTER(I)]
     lib.sp_strerror.argtypes = [I]
@@ -318,6 +320,15 @@ def sp_dense_pivot_attn_fixed_scratch(q, k, v, heads, block, out, importance_out
     _check(load().sp_dense_pivot_attn_fixed_scratch(dev, _view(q), _view(k), _view(v), _i32(heads), len(heads), block,
                                                     _view(out), _ptr(importance_out), _ptr(lse_out), _stream(stream)),
            "sp_dense_pivot_attn_fixed_scratch")
+
+
+def workspace_bytes_patterns(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots, pooled_construction=False):
+    """(bytes for sp_prefill_attn_auto, bytes for sp_prefill_attn_layer) at this problem size."""
+    a, b = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(load().sp_workspace_bytes_patterns(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivots,
+                                              int(bool(pooled_construction)), ctypes.byref(a), ctypes.byref(b)),
+           "sp_workspace_bytes_patterns")
+    return a.value, b.value
 
 
 def fixed_scratch_status(device=0):

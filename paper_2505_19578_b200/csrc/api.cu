@@ -177,6 +177,49 @@ WsLayout ws_layout(int Nb, int B, int n_pivots, bool paired) {
   return w;
 }
 
+// Workspace of sp_prefill_attn_auto and of sp_prefill_attn_layer (offsets in bytes, each 256-byte aligned).
+struct AutoLayout {
+  size_t imp, scores, mask, counts, indices, scratch, atilde, rows, small, vs, total;
+};
+AutoLayout auto_layout(const Problem& p, int n_pivots, int n_members, bool pooled, bool paired) {
+  AutoLayout w;
+  const size_t nn = (size_t)p.Nb * p.Nb;
+  const int lists = n_pivots + n_members;
+  const int rows = n_pivots > n_members ? n_pivots : n_members;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  w.imp = take(n_pivots * nn * (pooled ? sizeof(double) : sizeof(float)));   // importance, or the pooled map
+  w.scores = take(pooled ? n_pivots * nn * sizeof(float) : 0);
+  w.mask = take(lists * nn);
+  w.counts = take((size_t)lists * p.Nb * sizeof(int32_t));
+  w.indices = take(lists * nn * sizeof(int32_t));
+  w.scratch = take(pooled ? pooled_scratch_bytes(n_pivots, p.Nb, p.d) : stats_bytes(paired, n_pivots, p.Nb, p.B));
+  w.atilde = take((size_t)n_pivots * p.Nb * sizeof(float));
+  w.rows = take((size_t)rows * p.Nb * sizeof(double));
+  w.small = take((size_t)(3 * kMaxHeads + p.Hq) * sizeof(int32_t));
+  w.vs = take(vslash_scratch_bytes(n_members, p.N, 8));
+  w.total = off;
+  return w;
+}
+struct LayerLayout {
+  size_t ahat, rows, small, imp, scores, scratch, vs, total;
+};
+LayerLayout layer_layout(const Problem& p, int n_new_max, bool pooled, bool paired) {
+  LayerLayout w;
+  const size_t nn = (size_t)p.Nb * p.Nb;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  w.ahat = take((size_t)p.Hq * p.Nb * sizeof(float));
+  w.rows = take((size_t)p.Hq * p.Nb * sizeof(double));
+  w.small = take((size_t)(4 * kMaxHeads) * sizeof(int32_t) + (size_t)kMaxHeads * sizeof(float));
+  w.imp = take(n_new_max * nn * (pooled ? sizeof(double) : sizeof(float)));
+  w.scores = take(pooled ? nn * sizeof(float) : 0);
+  w.scratch = take(pooled ? pooled_scratch_bytes(n_new_max, p.Nb, p.d) : stats_bytes(paired, n_new_max, p.Nb, p.B));
+  w.vs = take(vslash_scratch_bytes(p.Hq, p.N, 8));
+  w.total = off;
+  return w;
+}
+
 __global__ void gather_masks_kernel(const uint8_t* __restrict__ pivot_masks, HeadTable src, int nb,
                                     uint8_t* __restrict__ out, const int32_t* __restrict__ src_dev = nullptr) {
   const int i = blockIdx.x, h = blockIdx.y;
@@ -248,6 +291,17 @@ int sp_workspace_bytes(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim,
   if (head_dim != 64 && head_dim != 128) return SP_ERR_UNSUPPORTED;
   if (seq % block != 0 || seq / block > kMaxNb || n_q_heads % n_kv_heads != 0) return SP_ERR_UNSUPPORTED;
   *bytes = ws_layout((int)(seq / block), block, n_pivots, goes_paired(0, head_dim, block)).total;
+  return SP_OK;
+}
+
+int sp_workspace_bytes_patterns(int64_t seq, int n_q_heads, int n_kv_heads, int head_dim, int block, int n_pivots,
+                                int pooled_construction, size_t* auto_bytes, size_t* layer_bytes) {
+  if (seq <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_pivots < 0 || n_pivots > n_q_heads) return SP_ERR_INVALID_ARG;
+  if (head_dim != 128 || block != 128) return SP_ERR_UNSUPPORTED;
+  if (seq % block != 0 || seq / block > kMaxNb || n_q_heads % n_kv_heads != 0 || n_q_heads > kMaxHeads) return SP_ERR_UNSUPPORTED;
+  Problem p{n_q_heads, n_kv_heads, (int)seq, head_dim, block, (int)(seq / block)};
+  if (auto_bytes) *auto_bytes = auto_layout(p, n_pivots, n_q_heads - n_pivots, pooled_construction != 0, true).total;
+  if (layer_bytes) *layer_bytes = layer_layout(p, n_pivots, pooled_construction != 0, true).total;
   return SP_OK;
 }
 
@@ -847,20 +901,9 @@ int sp_prefill_attn_auto(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, co
   // workspace
   const size_t nn = (size_t)p.Nb * p.Nb;
   const int n_lists = n_pivots + n_members;
-  const int n_row = n_pivots > n_members ? n_pivots : n_members;
-  size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
-  const size_t o_imp = take(n_pivots * nn * (pooled_construction ? sizeof(double) : sizeof(float)));   // importance, or the pooled map
-  const size_t o_scores = take(pooled_construction ? n_pivots * nn * sizeof(float) : 0);
-  const size_t o_mask = take(n_lists * nn);
-  const size_t o_counts = take((size_t)n_lists * p.Nb * sizeof(int32_t));
-  const size_t o_indices = take(n_lists * nn * sizeof(int32_t));
-  const size_t o_scratch = take(pooled_construction ? pooled_scratch_bytes(n_pivots, p.Nb, p.d)
-                                                    : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_pivots, p.Nb, p.B));
-  const size_t o_atilde = take((size_t)n_pivots * p.Nb * sizeof(float));
-  const size_t o_rows = take((size_t)n_row * p.Nb * sizeof(double));
-  const size_t o_small = take((size_t)(3 * kMaxHeads + p.Hq) * sizeof(int32_t));
-  const size_t o_vs = take(vslash_scratch_bytes(n_members, p.N, 8));
+  const AutoLayout w = auto_layout(p, n_pivots, n_members, pooled_construction != 0, goes_paired(ctx->kernel, p.d, p.B));
+  const size_t o_imp = w.imp, o_scores = w.scores, o_mask = w.mask, o_counts = w.counts, o_indices = w.indices,
+               o_scratch = w.scratch, o_atilde = w.atilde, o_rows = w.rows, o_small = w.small, o_vs = w.vs, off = w.total;
   if ((rc = reserve(ctx, off))) return rc;
   char* ws = static_cast<char*>(ctx->ws);
   float* imp = reinterpret_cast<float*>(ws + o_imp);
@@ -1030,16 +1073,9 @@ int sp_prefill_attn_layer(sp_ctx* ctx, sp_pattern_dict* dict, const sp_tensor* q
       if (c >= 0 && !dict->has[c] && !seen[c]) { seen[c] = 1; ++n_new_max; }
     }
   }
-  size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
-  const size_t o_ahat = take((size_t)p.Hq * p.Nb * sizeof(float));
-  const size_t o_rows = take((size_t)p.Hq * p.Nb * sizeof(double));
-  const size_t o_small = take((size_t)(4 * kMaxHeads) * sizeof(int32_t) + (size_t)kMaxHeads * sizeof(float));
-  const size_t o_imp = take(n_new_max * nn * (pooled_construction ? sizeof(double) : sizeof(float)));
-  const size_t o_scores = take(pooled_construction ? nn * sizeof(float) : 0);
-  const size_t o_scratch = take(pooled_construction ? pooled_scratch_bytes(n_new_max, p.Nb, p.d)
-                                                    : stats_bytes(goes_paired(ctx->kernel, p.d, p.B), n_new_max, p.Nb, p.B));
-  const size_t o_vs = take(vslash_scratch_bytes(p.Hq, p.N, 8));
+  const LayerLayout w = layer_layout(p, n_new_max, pooled_construction != 0, goes_paired(ctx->kernel, p.d, p.B));
+  const size_t o_ahat = w.ahat, o_rows = w.rows, o_small = w.small, o_imp = w.imp, o_scores = w.scores,
+               o_scratch = w.scratch, o_vs = w.vs, off = w.total;
   if ((rc = reserve(ctx, off))) return rc;
   char* ws = static_cast<char*>(ctx->ws);
   float* a_hat = reinterpret_cast<float*>(ws + o_ahat);

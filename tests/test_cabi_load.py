@@ -50,6 +50,9 @@ def test_host_only_calls(lib):
     # the one-row-block kernel (other shapes) keeps the per-tile layout
     b64 = binding.workspace_bytes(8192, 8, 8, 64, 64, 2)
     assert b64 >= 2 * 128 * 129 // 2 * 64 * 4
+    wa, wl = binding.workspace_bytes_patterns(131072, 32, 8, 128, 128, 6)
+    assert wa > 32 * nb * nb * 5 and wl > 0            # masks and lists of every head's own pattern
+    assert binding.workspace_bytes_patterns(131072, 32, 8, 128, 128, 6, True)[0] > wa - (200 << 20)
     out = ctypes.c_size_t()
     assert lib.sp_workspace_bytes(1000, 32, 8, 128, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED
     assert lib.sp_workspace_bytes(4096, 32, 8, 96, 128, 4, ctypes.byref(out)) == binding.SP_ERR_UNSUPPORTED
