@@ -18,7 +18,9 @@ extern "C" {
  * 128 the kernel that gives one CTA two adjacent row-blocks sharing their K/V
  * tiles, otherwise the one-row-block kernel), 1 = plain fp32 CUDA-core kernel
  * kept as an independent on-device cross-check, 2 = the one-row-block
- * tensor-core kernel for every shape. */
+ * tensor-core kernel for every shape, 3 = as 0, but every work item of the
+ * paired kernel is two adjacent row-blocks of one head (0 also gives one item
+ * to two heads of one KV head that walk the same list). */
 int sp_ctx_set_kernel(sp_ctx* ctx, int which);
 
 /* Phase trace of the tensor-core attention kernels (a profiling aid).  While a

@@ -160,7 +160,7 @@ class Context:
     __del__ = close
 
     def set_kernel(self, kernel: str):
-        _check(self._lib.sp_ctx_set_kernel(self._h, {"tc": 0, "simt": 1, "tc1": 2}[kernel]), "sp_ctx_set_kernel")
+        _check(self._lib.sp_ctx_set_kernel(self._h, {"tc": 0, "simt": 1, "tc1": 2, "tc_single_head_items": 3}[kernel]), "sp_ctx_set_kernel")
 
     def set_trace(self, events, events_per_role: int):
         """events: zeroed CUDA int64 tensor of 5 * events_per_role * 2 entries, or None to switch off."""

@@ -120,6 +120,7 @@ AttnArgs base_args(const sp_ctx* ctx, const Problem& p, const sp_tensor* q, cons
   a.work_counter = ctx->status ? ctx->status + 2 : nullptr;
   a.trace = ctx->trace;
   a.trace_cap = ctx->trace_cap;
+  a.pair_heads = ctx->kernel != 3;
   a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)p.d));
   return a;
 }
@@ -146,7 +147,7 @@ int launch_attn(sp_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   if (a.n_heads == 0) return SP_OK;
   cudaError_t e;
   if (ctx->kernel == 1) e = launch_attn_simt(a, s);
-  else if (ctx->kernel == 0 && attn_pair_supported(a)) e = launch_attn_pair(a, s);
+  else if ((ctx->kernel == 0 || ctx->kernel == 3) && attn_pair_supported(a)) e = launch_attn_pair(a, s);
   else e = launch_attn_tc(a, s);
   if (e != cudaSuccess) return SP_ERR_CUDA;
   ctx->launches += 1;
@@ -155,7 +156,7 @@ int launch_attn(sp_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
 
 // Bytes of tile statistics a dense launch over n_heads heads with importance needs.  `paired`: the launch goes to the
 // paired kernel (one region per CTA, used by every launch in turn); otherwise one region per head.
-bool goes_paired(int kernel, int d, int B) { return kernel == 0 && d == 128 && B == 128; }
+bool goes_paired(int kernel, int d, int B) { return (kernel == 0 || kernel == 3) && d == 128 && B == 128; }
 size_t stats_bytes(bool paired, int n_heads, int Nb, int B) {
   return paired ? attn_pair_stats_bytes(n_heads, Nb) : (size_t)n_heads * tile_stats_bytes_per_head(Nb, B);
 }
@@ -335,7 +336,7 @@ int sp_selftest_wait_timeout(sp_ctx* ctx, int64_t limit_cycles, void* stream) {
 }
 
 int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
-  if (!ctx || which < 0 || which > 2) return SP_ERR_INVALID_ARG;
+  if (!ctx || which < 0 || which > 3) return SP_ERR_INVALID_ARG;
   ctx->kernel = which;
   return SP_OK;
 }

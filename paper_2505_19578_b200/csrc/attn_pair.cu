@@ -6,8 +6,10 @@
 //   probability mass of each (query-block, key-block) tile; a member walks the
 //   compacted list of key-blocks its cluster's pivot selected.
 //
-// Persistent CTAs, one per SM.  A work item is one head and TWO adjacent query
-// row-blocks (tile A = row-block 2u, tile B = row-block 2u+1), 256 query rows.
+// Persistent CTAs, one per SM.  A work item is TWO tiles of 128 query rows that
+// read the same KV head: two adjacent row-blocks of one head (tile A = row-block
+// 2u, tile B = row-block 2u+1) or, where two heads of one KV head walk the same
+// list (two members of a cluster, two dense heads), the same row-block of both.
 // The items of a launch are ordered (the heads of one KV head together, the
 // longest pairs first) and handed out through a device counter, so an SM that
 // finishes early takes the next item; barriers and tensor memory are set up once
@@ -15,8 +17,9 @@
 // softmax warps still write out the item before.  The two tiles walk the UNION
 // of their key-block lists in ascending order, so a K/V tile both of them need
 // is brought into shared memory once and feeds four MMAs instead of two; a
-// key-block only one of them selected is computed for that tile alone.  (Dense:
-// the union is 0..2u+1, the last key-block is B's diagonal tile only.)
+// key-block only one of them selected is computed for that tile alone.  (Dense,
+// one head: the union is 0..2u+1, the last key-block is B's diagonal tile only.
+// Two heads on one list: the lists are equal and every K/V tile serves both.)
 //
 // Warp roles (320 threads):
 //   warps 0-3   softmax of tile A: thread t owns query row t = TMEM lane t
@@ -255,16 +258,20 @@ __device__ __forceinline__ void issue_pv_c(bool accumulate) {   // O_X (+)= P_X 
     mma_ts(kOCol + X * 128, kSCol + X * 128 + kk * 8, dv + (uint32_t)((kk * 16 * 128) >> 4), idesc, (accumulate || kk > 0) ? 1u : 0u);
 }
 
-// One work item as the scheduler warp posts it to the other roles (shared memory, two slots of eight ints).
+// One work item as the producer warp posts it to the other roles (shared memory, two slots of sixteen ints).
 struct Item {
-  int id;      // position in the work order, -1 = no more work
-  int slot;    // position of the head in the call's head table
-  int u;       // pair of row-blocks 2u, 2u + 1
-  int h;       // query head
-  int list;    // list index, -1 = dense
-  int cntA;    // key-blocks tile A visits
-  int cntB;    // key-blocks tile B visits
+  int id;              // position in the work order, -1 = no more work
+  int slotA, slotB;    // position of each tile's head in the call's head table
+  int hA, hB;          // query head of each tile (both read the same KV head)
+  int iA, iB;          // row-block of each tile (>= Nb: the tile does not exist)
+  int listA, listB;    // list index of each tile, -1 = dense
+  int cntA, cntB;      // key-blocks each tile visits
 };
+enum { ITEM_INTS = 16 };
+// An entry of the work order: one head (tile A = row-block 2u, tile B = row-block 2u + 1 of that head), or two heads of
+// one KV head that walk the same list (tile A = row-block i of the first, tile B = row-block i of the second; one entry
+// for the even i, one for the odd i, so that every entry has ceil(Nb / 2) items).
+enum { ENT_ONE_HEAD = 0, ENT_TWO_HEADS_EVEN = 1, ENT_TWO_HEADS_ODD = 2 };
 
 // Rare path of the softmax, kept out of the hot loop: the row's reference max has moved, so O of the earlier
 // steps (when there are any) and the P chunks of this key-block that are already stored are brought to the new
@@ -319,7 +326,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kMiscOff + 260);
   volatile int* kflags = reinterpret_cast<volatile int*>(smem + kMiscOff + 264);   // [kStages]
   float* lse_smem = reinterpret_cast<float*>(smem + kMiscOff + 512);               // [2][128]
-  volatile int* items = reinterpret_cast<volatile int*>(smem + kMiscOff + 1536);   // [2][8]
+  volatile int* items = reinterpret_cast<volatile int*>(smem + kMiscOff + 1536);   // [2][ITEM_INTS]
   auto bar = [&](int which) { return smem_u32(bars + which); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -367,13 +374,13 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
   auto take_item = [&](int k, Item& it, int where) -> bool {
     const int sl = k & 1;
     if (!__all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_FULL + sl), (uint32_t)(k >> 1) & 1u, ab, where))) return false;
-    it.id = items[8 * sl + 0];
-    it.slot = items[8 * sl + 1];
-    it.u = items[8 * sl + 2];
-    it.h = items[8 * sl + 3];
-    it.list = items[8 * sl + 4];
-    it.cntA = items[8 * sl + 5];
-    it.cntB = items[8 * sl + 6];
+    const volatile int* src = items + ITEM_INTS * sl;
+    it.id = src[0];
+    it.slotA = src[1]; it.slotB = src[2];
+    it.hA = src[3]; it.hB = src[4];
+    it.iA = src[5]; it.iB = src[6];
+    it.listA = src[7]; it.listB = src[8];
+    it.cntA = src[9]; it.cntB = src[10];
     __syncwarp();
     if (lane == 0) mbar_arrive(bar(BAR_ITEM_EMPTY + sl));
     return true;
@@ -399,7 +406,7 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           const int sl = k & 1;
           if (k >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_ITEM_EMPTY + sl), ((uint32_t)(k >> 1) & 1u) ^ 1u, ab, 40));
           if (!ok) break;
-          it.id = -1; it.slot = 0; it.u = 0; it.h = 0; it.list = -1; it.cntA = 0; it.cntB = 0;
+          it.id = -1; it.slotA = it.slotB = 0; it.hA = it.hB = 0; it.iA = it.iB = 0; it.listA = it.listB = -1; it.cntA = it.cntB = 0;
           if (lane == 0) {
             const int raw = poisoned ? n_items : atomicAdd(a.work_counter, 1);
             if (raw < n_items) {
@@ -409,20 +416,27 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
                 ++g;
               }
               const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
+              const int ent = a.order.v[a.group_start.v[g] + rest % ng];
+              const int u = n_pairs - 1 - rest / ng;
+              const int kind = ent >> 16;
               it.id = raw;
-              it.slot = a.order.v[a.group_start.v[g] + rest % ng];
-              it.u = n_pairs - 1 - rest / ng;
-              it.slot = sp_in_range(it.slot, 0, a.n_heads - 1, a.status, 51);
-              it.h = sp_in_range(a.heads.v[it.slot], 0, a.n_q_heads - 1, a.status, 51);
-              it.list = a.lists_dev ? a.lists_dev[it.slot] : a.lists.v[it.slot];
-              if (it.list < 0) it.list = -1;
+              it.slotA = sp_in_range(ent & 0xff, 0, a.n_heads - 1, a.status, 51);
+              it.slotB = sp_in_range((ent >> 8) & 0xff, 0, a.n_heads - 1, a.status, 51);
+              it.iA = kind == ENT_ONE_HEAD ? 2 * u : 2 * u + (kind - ENT_TWO_HEADS_EVEN);
+              it.iB = kind == ENT_ONE_HEAD ? 2 * u + 1 : it.iA;
+              it.hA = sp_in_range(a.heads.v[it.slotA], 0, a.n_q_heads - 1, a.status, 51);
+              it.hB = sp_in_range(a.heads.v[it.slotB], 0, a.n_q_heads - 1, a.status, 51);
+              it.listA = a.lists_dev ? a.lists_dev[it.slotA] : a.lists.v[it.slotA];
+              it.listB = a.lists_dev ? a.lists_dev[it.slotB] : a.lists.v[it.slotB];
+              if (it.listA < 0) it.listA = -1;
+              if (it.listB < 0) it.listB = -1;
               int cnt[2];
 #pragma unroll
               for (int x = 0; x < 2; ++x) {
-                const int i = 2 * it.u + x;
+                const int i = x ? it.iB : it.iA, list = x ? it.listB : it.listA;
                 int c = 0;
                 if (i < a.Nb) {
-                  c = it.list >= 0 ? a.counts[(size_t)it.list * a.Nb + i] : i + 1;
+                  c = list >= 0 ? a.counts[(size_t)list * a.Nb + i] : i + 1;
                   c = c < 0 ? 0 : (c > i + 1 ? i + 1 : c);
                 }
                 cnt[x] = c;
@@ -430,60 +444,63 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
               it.cntA = cnt[0];
               it.cntB = cnt[1];
             }
-            items[8 * sl + 0] = it.id;
-            items[8 * sl + 1] = it.slot;
-            items[8 * sl + 2] = it.u;
-            items[8 * sl + 3] = it.h;
-            items[8 * sl + 4] = it.list;
-            items[8 * sl + 5] = it.cntA;
-            items[8 * sl + 6] = it.cntB;
+            volatile int* dst = items + ITEM_INTS * sl;
+            dst[0] = it.id;
+            dst[1] = it.slotA; dst[2] = it.slotB;
+            dst[3] = it.hA; dst[4] = it.hB;
+            dst[5] = it.iA; dst[6] = it.iB;
+            dst[7] = it.listA; dst[8] = it.listB;
+            dst[9] = it.cntA; dst[10] = it.cntB;
             mbar_arrive(bar(BAR_ITEM_FULL + sl));
           }
           it.id = __shfl_sync(0xffffffffu, it.id, 0);
-          it.u = __shfl_sync(0xffffffffu, it.u, 0);
-          it.h = __shfl_sync(0xffffffffu, it.h, 0);
-          it.list = __shfl_sync(0xffffffffu, it.list, 0);
+          it.hA = __shfl_sync(0xffffffffu, it.hA, 0);
+          it.hB = __shfl_sync(0xffffffffu, it.hB, 0);
+          it.iA = __shfl_sync(0xffffffffu, it.iA, 0);
+          it.iB = __shfl_sync(0xffffffffu, it.iB, 0);
+          it.listA = __shfl_sync(0xffffffffu, it.listA, 0);
+          it.listB = __shfl_sync(0xffffffffu, it.listB, 0);
           it.cntA = __shfl_sync(0xffffffffu, it.cntA, 0);
           it.cntB = __shfl_sync(0xffffffffu, it.cntB, 0);
         }
         if (it.id < 0) break;
         const int cntA = it.cntA, cntB = it.cntB;
         if (cntA + cntB == 0) continue;
-        const int iA = 2 * it.u, iB = iA + 1;
-        const int g = it.h / a.group;
+        const int iA = it.iA, iB = it.iB;
+        const int g = it.hA / a.group;     // tile B's head reads the same KV head
         // Q of the item before this one has been read by its last QK^T
         if (qn > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_Q_EMPTY), (uint32_t)(qn - 1) & 1u, ab, 15));
         if (!ok) break;
         if (lane == 0) {
-          const int n_q = iB < a.Nb ? 2 : 1;
+          const int n_q = iB < a.Nb ? 2 : 1;     // tile A exists whenever the item has work
           mbar_expect_tx(bar(BAR_Q_FULL), n_q * kTile);
           for (int x = 0; x < n_q; ++x)
             for (int b = 0; b < 2; ++b)
-              tma_load_3d(sQ + b * kTile + x * kBox, &tm_q, bar(BAR_Q_FULL), b * 64, (iA + x) * BLK, it.h);
+              tma_load_3d(sQ + b * kTile + x * kBox, &tm_q, bar(BAR_Q_FULL), b * 64, (x ? iB : iA) * BLK, x ? it.hB : it.hA);
         }
         ++qn;
         // The two ascending lists are merged 32 entries at a time: lane l holds entry base + l.
-        const int32_t* idxA = it.list >= 0 ? a.indices + ((size_t)it.list * a.Nb + iA) * a.Nb : nullptr;
-        const int32_t* idxB = it.list >= 0 && iB < a.Nb ? a.indices + ((size_t)it.list * a.Nb + iB) * a.Nb : nullptr;
+        const int32_t* idxA = it.listA >= 0 && iA < a.Nb ? a.indices + ((size_t)it.listA * a.Nb + iA) * a.Nb : nullptr;
+        const int32_t* idxB = it.listB >= 0 && iB < a.Nb ? a.indices + ((size_t)it.listB * a.Nb + iB) * a.Nb : nullptr;
         int pa = 0, pb = 0, n = 0;
         int chunkA = 0, chunkB = 0;
         if (idxA) chunkA = lane < cntA ? idxA[lane] : 0;
         if (idxB) chunkB = lane < cntB ? idxB[lane] : 0;
-        const bool listed = it.list >= 0;
+        const bool listedA = idxA != nullptr, listedB = idxB != nullptr;
         while ((pa < cntA || pb < cntB) && ok) {
-          const int ja = pa < cntA ? (listed ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
-          const int jb = pb < cntB ? (listed ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
+          const int ja = pa < cntA ? (listedA ? __shfl_sync(0xffffffffu, chunkA, pa & 31) : pa) : 0x7fffffff;
+          const int jb = pb < cntB ? (listedB ? __shfl_sync(0xffffffffu, chunkB, pb & 31) : pb) : 0x7fffffff;
           const int j_listed = ja < jb ? ja : jb;
           int f = (ja == j_listed ? F_A : 0) | (jb == j_listed ? F_B : 0);
-          // a listed key-block lies on or before the diagonal of the later tile that walks it
-          const int j = sp_in_range(j_listed, 0, (f & F_B) ? iB : iA, a.status, 50);
+          // a listed key-block lies on or before the diagonal of every tile that walks it
+          const int j = sp_in_range(j_listed, 0, (f & F_A) ? ((f & F_B) && iB < iA ? iB : iA) : iB, a.status, 50);
           if (ja == j_listed) {
             ++pa;
-            if (listed && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
+            if (listedA && (pa & 31) == 0) chunkA = pa + lane < cntA ? idxA[pa + lane] : 0;
           }
           if (jb == j_listed) {
             ++pb;
-            if (listed && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
+            if (listedB && (pb & 31) == 0) chunkB = pb + lane < cntB ? idxB[pb + lane] : 0;
           }
           if (!(pa < cntA || pb < cntB)) f |= F_LAST;
           const int gn = gk + n;
@@ -659,10 +676,10 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
       // by the epilogue of the item before from the writes of this item.
       if (!bar_and(1 + x, 128, got)) break;
       if (it.id < 0) break;
-      const int i = 2 * it.u + x, cnt = x ? it.cntB : it.cntA;
-      const int h = it.h, slot = it.slot;
-      const int32_t* idx = it.list >= 0 && i < a.Nb ? a.indices + ((size_t)it.list * a.Nb + i) * a.Nb : nullptr;
-      const bool emit = a.importance != nullptr && it.list < 0;
+      const int i = x ? it.iB : it.iA, cnt = x ? it.cntB : it.cntA;
+      const int h = x ? it.hB : it.hA, slot = x ? it.slotB : it.slotA, list = x ? it.listB : it.listA;
+      const int32_t* idx = list >= 0 && i < a.Nb ? a.indices + ((size_t)list * a.Nb + i) * a.Nb : nullptr;
+      const bool emit = a.importance != nullptr && list < 0;
       const int r = i * BLK + row;
       float m_ref = -CUDART_INF_F, l = 0.f;
       bool ok = cnt > 0;
@@ -871,21 +888,48 @@ cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
   // Work order.  Many items (forty per SM or more): the slots sorted by KV head (stable), one group per KV head,
   // so that a K/V set stays in L2 while its heads run.  Fewer: one group, i.e. the longest pairs of all heads
   // first, because then the balance at the end matters more than L2.
+  // Two heads of one KV head that walk the same list (members of one cluster; two dense heads) share a work item
+  // row-block by row-block: their two tiles need exactly the same K/V tiles, so no K/V load serves one tile alone,
+  // as happens wherever two adjacent row-blocks of one head differ in their lists.  Such a pair takes two entries
+  // (even and odd row-blocks); a head without a partner keeps one entry and pairs its own adjacent row-blocks.
+  // Lists decided on the device are not known here: those heads stay single.
   const int n_sm = sm_count();
   const bool by_kv_head = (long)a.n_heads * ((a.Nb + 1) / 2) >= 40L * n_sm;
   int n = 0;
   a.n_groups = 0;
+  bool taken[kMaxHeads];
+  for (int t = 0; t < a.n_heads; ++t) taken[t] = false;
+  auto add_head = [&](int t) {
+    if (taken[t]) return;
+    taken[t] = true;
+    int partner = -1;
+    if (!a.lists_dev && a.pair_heads) {
+      const int lt = a.lists.v[t] < 0 ? -1 : a.lists.v[t];
+      for (int t2 = t + 1; t2 < a.n_heads && partner < 0; ++t2) {
+        const int l2 = a.lists.v[t2] < 0 ? -1 : a.lists.v[t2];
+        if (!taken[t2] && a.heads.v[t2] / a.group == a.heads.v[t] / a.group && l2 == lt && a.heads.v[t2] != a.heads.v[t]) partner = t2;
+      }
+    }
+    if (partner >= 0) {
+      taken[partner] = true;
+      a.order.v[n++] = t | (partner << 8) | (ENT_TWO_HEADS_EVEN << 16);
+      a.order.v[n++] = t | (partner << 8) | (ENT_TWO_HEADS_ODD << 16);
+    } else {
+      a.order.v[n++] = t | (t << 8) | (ENT_ONE_HEAD << 16);
+    }
+  };
   if (by_kv_head) {
     for (int g = 0; g < a.n_kv_heads; ++g) {
       const int start = n;
       for (int t = 0; t < a.n_heads; ++t)
-        if (a.heads.v[t] / a.group == g) a.order.v[n++] = t;
+        if (a.heads.v[t] / a.group == g) add_head(t);
       if (n > start) a.group_start.v[a.n_groups++] = start;
     }
   } else {
-    for (int t = 0; t < a.n_heads; ++t) a.order.v[n++] = t;
+    for (int t = 0; t < a.n_heads; ++t) add_head(t);
     a.group_start.v[a.n_groups++] = 0;
   }
+  static_assert(kMaxHeads <= 256, "an entry of the work order holds two slots of eight bits");
   static_assert(sizeof(a.group_start.v) / sizeof(a.group_start.v[0]) == kMaxHeads + 1, "room for the end of the last group");
   a.group_start.v[a.n_groups] = n;
   CUtensorMap tq, tk, tv;

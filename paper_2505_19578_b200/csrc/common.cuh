@@ -61,6 +61,7 @@ struct AttnArgs {
   int* work_counter;       // paired kernel: device int, the launch's position in its work order (cleared by the launcher)
   long long* trace;        // optional phase trace of CTA (0,0): 5 roles x trace_cap x {tag, clock}
   int trace_cap;
+  int pair_heads;          // paired kernel: heads of one KV head that walk the same list share work items (launcher)
   float scale_log2;        // log2(e) / sqrt(d)
 };
 

@@ -174,6 +174,61 @@ def test_block_sparse_attn_matches_oracle(binding, kernel, Hq, Hkv, N, d, B):
         par.assert_out_close(par.f64(out[h]), ref, f"head {h}")
 
 
+def test_two_heads_of_one_kv_head_share_work_items(binding):
+    """Heads of one KV head that walk the same list are given common work items (tile A = a row-block of one head, tile B
+    = the same row-block of the other).  Every tile still walks its own list in the same order, so the result is the same
+    bit for bit as with one head per item, and it matches the oracle.  11 row-blocks: the odd tail; five heads of one
+    KV head on two lists and dense: two pairs and one head left over."""
+    Hq, Hkv, N, d, B = 6, 1, 1408, 128, 128
+    q, k, v = _rand_layer(17, Hq, Hkv, N, d)
+    Q, K, V = par.f64(q), par.f64(k), par.f64(v)
+    Nb = N // B
+    rng = np.random.default_rng(9)
+    masks = np.zeros((2, Nb, Nb), np.uint8)
+    for l in range(2):
+        m = np.tril(rng.random((Nb, Nb)) < 0.4).astype(np.uint8)
+        for i in range(Nb):
+            if m[i].sum() == 0:
+                m[i, rng.integers(0, i + 1)] = 1
+        masks[l] = m
+    counts = torch.from_numpy(masks.sum(axis=2).astype(np.int32)).cuda()
+    indices = np.full((2, Nb, Nb), -1, np.int32)
+    for l in range(2):
+        for i in range(Nb):
+            sel = np.nonzero(masks[l, i])[0]
+            indices[l, i, :len(sel)] = sel
+    indices = torch.from_numpy(indices).cuda()
+    heads = [4, 0, 3, 5, 1, 2]
+    lists = [1, 0, 1, -1, 1, -1]        # list 1: heads 4 and 3 together, head 1 alone; dense: heads 5 and 2 together
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    outs = {}
+    for kern in ("tc", "tc_single_head_items"):
+        ctx = binding.Context(kernel=kern)
+        out = torch.full((Hq, N, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ctx.sp_block_sparse_attn(qc, kc, vc, heads, lists, counts, indices, B, out)
+        _sync_ok(ctx)
+        outs[kern] = out
+    assert torch.equal(outs["tc"], outs["tc_single_head_items"])
+    for h, l in zip(heads, lists):
+        M = masks[l] if l >= 0 else np.tril(np.ones((Nb, Nb), np.uint8))
+        par.assert_out_close(par.f64(outs["tc"][h]), orc.masked_attention(Q, K, V, h, M, B), f"head {h}")
+    # dense with the importance map: the three heads 5, 2, 0 of the KV head -> one pair and one head alone
+    imps = {}
+    for kern in ("tc", "tc_single_head_items"):
+        ctx = binding.Context(kernel=kern)
+        out = torch.zeros((Hq, N, d), dtype=torch.bfloat16, device="cuda")
+        imp = torch.full((3, Nb, Nb), float("nan"), device="cuda")
+        ctx.sp_dense_pivot_attn(qc, kc, vc, [5, 2, 0], B, out, importance_out=imp)
+        _sync_ok(ctx)
+        imps[kern] = (out, imp)
+    assert torch.equal(imps["tc"][0], imps["tc_single_head_items"][0])
+    assert torch.equal(imps["tc"][1], imps["tc_single_head_items"][1])
+    for t, h in enumerate([5, 2, 0]):
+        imp_ref, o_ref = orc.importance_map(Q, K, V, h, B)
+        par.assert_out_close(par.f64(imps["tc"][0][h]), o_ref, f"dense head {h}")
+        np.testing.assert_allclose(imps["tc"][1][t].cpu().numpy(), imp_ref, rtol=0, atol=par.IMP_ATOL)
+
+
 # ------------------------------------------------------------------ the whole layer
 
 _run_layer = par.run_layer
