@@ -626,14 +626,19 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
   // this context may still be reading the device copies).
   if (!hand_over(sc, sin) || !hand_over(sc, sout)) return SP_ERR_CUDA;
 
-  // Order of the work (and, with it, of the copies in): every pivot but the last — the first of them alone (its
-  // KV head and its queries in, step 1, its output out), so that computing starts after three heads' worth of
-  // bytes, the others in one launch; then the other KV heads, step 2 for those pivots and their clusters'
-  // members in groups (queries in, step 4, outputs out); then the last pivot and its cluster.  With every pivot
-  // first the copies out have nothing to carry for the first half of the call and trail the last kernel by a
-  // quarter of it; with the last pivot held back they overlap the members' attention, and what follows the last
-  // copy in is one cluster.  (Measured at 128K, 32 query heads: 41.5 ms with all pivots in one launch first, 38.4
-  // with one pivot per launch, 37.8 with the last pivot held back, 37.6 in this order; the copies in alone take 29 ms.)
+  // Order of the work (and, with it, of the copies in): cluster by cluster, the pivots one cluster ahead.  For a
+  // pivot: its KV head (if not yet on the device) and its queries in, step 1 and step 2 for it alone, its output out;
+  // for its cluster's members, in groups of one or two heads: their KV heads and queries in, step 4, outputs out.
+  // Sequence: pivot 0, pivot 1, members 0, pivot 2, members 1, ..., members n-2, members n-1.  The copies in are the
+  // longest resource of the call (1.6 GB against 1.1 GB out and 25 ms of kernels at 128K with 32 query heads; with the
+  // copies out running beside them they take 32 ms), so the call cannot end before they do; what has to be kept short
+  // is what follows the last copy in, and the copies out must have work from early on.  With every pivot first they
+  // have nothing to carry for the first half of the call and trail the last kernel by a quarter of it; with a pivot
+  // right before its own cluster the members whose bytes came in during its step 1 (3.5 ms) leave a backlog of outputs
+  // behind the last pivot that outlasts the copies in by 3 ms.  One cluster ahead, the last pivot is through while a
+  // whole cluster of members is still to come in, and the tail is one head's kernel and the backlog of two or three
+  // outputs.  (Measured at 128K: 41.5 ms all pivots in one launch first, 38.4 one pivot per launch first, 35.6 the last
+  // pivot and its cluster at the end or cluster by cluster, 34.3 in this order; the copies in alone take 29 ms.)
   const char* hk = static_cast<const char*>(k_host);
   const char* hv = static_cast<const char*>(v_host);
   auto copy_in_kv = [&](int gkv) {
@@ -645,36 +650,24 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
   const int group = n_q_heads / n_kv_heads;
   const size_t stats_floats_per_head = tile_stats_bytes_per_head(p.Nb, p.B) / sizeof(float);
   const size_t nn = (size_t)p.Nb * p.Nb;
-  // steps 1 and 2 for the pivots t0 .. t1-1
-  auto run_pivots = [&](int t0, int t1) -> int {
-    // the first pivot of the range alone (so that computing starts after one pivot's bytes), the others in one
-    // launch (their bytes land while the first one computes, and one launch of several heads balances its last
-    // wave better than several one-head launches: 4 x 4.4 ms against 15.7 ms for four heads at 128K)
-    for (int u0 = t0; u0 < t1;) {
-      const int u1 = u0 == t0 ? u0 + 1 : t1;
-      for (int t = u0; t < u1; ++t) {
-        const int gkv = pivot_heads[t] / group;
-        if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return SP_ERR_CUDA; kv_sent[gkv] = true; }
-        if (!copy_in_head(pivot_heads[t])) return SP_ERR_CUDA;
-      }
-      if (!hand_over(sin, sc)) return SP_ERR_CUDA;
-      AttnArgs a = base_args(ctx, p, &q, &k, &v, &o);
-      a.n_heads = u1 - u0;
-      for (int t = u0; t < u1; ++t) { a.heads.v[t - u0] = pivot_heads[t]; a.lists.v[t - u0] = -1; }
-      a.importance = imp + (size_t)u0 * nn;
-      a.tile_stats = paired ? stats : stats + (size_t)u0 * stats_floats_per_head;   // launches on one stream take turns
-      if (int r = launch_attn(ctx, a, sc)) return r;
-      if (!hand_over(sc, sout)) return SP_ERR_CUDA;
-      for (int t = u0; t < u1; ++t)
-        if (!copy_out_head(pivot_heads[t])) return SP_ERR_CUDA;
-      u0 = u1;
-    }
-    if (t1 > t0) {
-      MaskArgs m{imp + (size_t)t0 * nn, t1 - t0, p.Nb, (double)gamma, pmask + (size_t)t0 * nn, counts + (size_t)t0 * p.Nb,
-                 indices + (size_t)t0 * nn};
-      if (launch_block_mask(m, sc) != cudaSuccess) return SP_ERR_CUDA;
-      ctx->launches += 1;
-    }
+  // steps 1 and 2 for pivot t alone
+  auto run_pivot = [&](int t) -> int {
+    const int gkv = pivot_heads[t] / group;
+    if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return SP_ERR_CUDA; kv_sent[gkv] = true; }
+    if (!copy_in_head(pivot_heads[t])) return SP_ERR_CUDA;
+    if (!hand_over(sin, sc)) return SP_ERR_CUDA;
+    AttnArgs a = base_args(ctx, p, &q, &k, &v, &o);
+    a.n_heads = 1;
+    a.heads.v[0] = pivot_heads[t];
+    a.lists.v[0] = -1;
+    a.importance = imp + (size_t)t * nn;
+    a.tile_stats = paired ? stats : stats + (size_t)t * stats_floats_per_head;   // launches on one stream take turns
+    if (int r = launch_attn(ctx, a, sc)) return r;
+    if (!hand_over(sc, sout)) return SP_ERR_CUDA;
+    if (!copy_out_head(pivot_heads[t])) return SP_ERR_CUDA;
+    MaskArgs m{imp + (size_t)t * nn, 1, p.Nb, (double)gamma, pmask + (size_t)t * nn, counts + (size_t)t * p.Nb, indices + (size_t)t * nn};
+    if (launch_block_mask(m, sc) != cudaSuccess) return SP_ERR_CUDA;
+    ctx->launches += 1;
     return SP_OK;
   };
   HeadTable mask_src;
@@ -687,27 +680,38 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
     member_list[n_members] = t;
     ++n_members;
   }
-  // step 4 for the members whose list is one of t0 .. t1-1 (and, with t0 == 0, for those that run dense), in
-  // groups; `shrink`: the groups become single heads towards the end, so that little is left after the last copy in
-  auto run_members = [&](int t0, int t1, bool shrink) -> int {
+  // step 4 for the members whose list is t (t < 0: those that run dense), in groups of two heads of one KV head
+  // where there are such (they share work items when they walk one list), else of one; `last`: nothing follows, so
+  // the last few heads go singly (what remains after the last copy in is then one head's kernel and copy out)
+  auto run_members = [&](int t, bool last) -> int {
     int sel[kMaxHeads], n_sel = 0;
     for (int x = 0; x < n_members; ++x)
-      if ((member_list[x] >= t0 && member_list[x] < t1) || (t0 == 0 && member_list[x] < 0)) sel[n_sel++] = x;
-    for (int g0 = 0, g1 = 0; g0 < n_sel; g0 = g1) {
-      const int left = n_sel - g0;
-      g1 = g0 + (!shrink || left > 8 ? (left < 4 ? left : 4) : left > 4 ? 2 : 1);
-      for (int x = g0; x < g1; ++x)
-        if (!copy_in_head(members[sel[x]])) return SP_ERR_CUDA;
+      if (member_list[x] == t || (t < 0 && member_list[x] < 0)) sel[n_sel++] = x;
+    bool done[kMaxHeads];
+    for (int x = 0; x < n_sel; ++x) done[x] = false;
+    for (int x0 = 0; x0 < n_sel; ++x0) {
+      if (done[x0]) continue;
+      int grp[2] = {sel[x0], -1}, n_grp = 1;
+      done[x0] = true;
+      int left = 0;
+      for (int x1 = x0 + 1; x1 < n_sel; ++x1) left += done[x1] ? 0 : 1;
+      for (int x1 = x0 + 1; x1 < n_sel && n_grp < 2 && (!last || left > 3); ++x1)
+        if (!done[x1] && members[sel[x1]] / group == members[sel[x0]] / group) { grp[n_grp++] = sel[x1]; done[x1] = true; }
+      for (int y = 0; y < n_grp; ++y) {
+        const int gkv = members[grp[y]] / group;
+        if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return SP_ERR_CUDA; kv_sent[gkv] = true; }
+        if (!copy_in_head(members[grp[y]])) return SP_ERR_CUDA;
+      }
       if (!hand_over(sin, sc)) return SP_ERR_CUDA;
       AttnArgs b = base_args(ctx, p, &q, &k, &v, &o);
       b.counts = counts;
       b.indices = indices;
-      b.n_heads = g1 - g0;
-      for (int x = g0; x < g1; ++x) { b.heads.v[x - g0] = members[sel[x]]; b.lists.v[x - g0] = member_list[sel[x]]; }
+      b.n_heads = n_grp;
+      for (int y = 0; y < n_grp; ++y) { b.heads.v[y] = members[grp[y]]; b.lists.v[y] = member_list[grp[y]]; }
       if (int r = launch_attn(ctx, b, sc)) return r;
       if (!hand_over(sc, sout)) return SP_ERR_CUDA;
-      for (int x = g0; x < g1; ++x)
-        if (!copy_out_head(members[sel[x]])) return SP_ERR_CUDA;
+      for (int y = 0; y < n_grp; ++y)
+        if (!copy_out_head(members[grp[y]])) return SP_ERR_CUDA;
     }
     return SP_OK;
   };
@@ -719,15 +723,15 @@ int sp_prefill_attn_host(sp_ctx* ctx, const void* q_host, const void* k_host, co
     hand_over(sin, sc);
     return code;
   };
-  const int n_first = n_pivots > 1 ? n_pivots - 1 : n_pivots;
-  if ((rc = run_pivots(0, n_first))) return bail(rc);
-  for (int gkv = 0; gkv < n_kv_heads; ++gkv)
-    if (!kv_sent[gkv]) { if (!copy_in_kv(gkv)) return bail(SP_ERR_CUDA); kv_sent[gkv] = true; }
-  if (!hand_over(sin, sc)) return bail(SP_ERR_CUDA);                             // members read every KV head
-  if ((rc = run_members(0, n_first, n_first == n_pivots))) return bail(rc);
-  if (n_first < n_pivots) {
-    if ((rc = run_pivots(n_first, n_pivots))) return bail(rc);
-    if ((rc = run_members(n_first, n_pivots, true))) return bail(rc);
+  // heads of clusters without a pivot run dense and wait for nothing: first (a head's dense attention takes five times
+  // as long as the copy of its output, so at the end of the call it would leave the copies out idle)
+  if ((rc = run_members(-1, n_pivots == 0))) return bail(rc);
+  // the pivots run one cluster ahead of the members: when the members of cluster t are through, the pattern of
+  // cluster t + 1 is there and its members follow at once, and nothing but members follows the last pivot
+  if (n_pivots > 0 && (rc = run_pivot(0))) return bail(rc);
+  for (int t = 0; t < n_pivots; ++t) {
+    if (t + 1 < n_pivots && (rc = run_pivot(t + 1))) return bail(rc);
+    if ((rc = run_members(t, t == n_pivots - 1))) return bail(rc);
   }
   if (mask_out_host) {
     gather_masks_kernel<<<dim3(p.Nb, p.Hq), 128, 0, sc>>>(pmask, mask_src, p.Nb, dmask);
