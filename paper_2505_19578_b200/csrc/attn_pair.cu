@@ -50,13 +50,16 @@
 // and is the TMEM A operand of PV; the next QK of that tile is issued after the
 // PV that reads P, and the tensor pipe keeps issue order.
 //
-// What bounds the kernel is the issuing warp.  The tensor pipe accepts an MMA
-// only a couple of instructions ahead, and the issuing thread needs about twenty
-// dependent instructions per tcgen05.mma (election, moves into uniform
-// registers), on a scheduler it shares with two softmax warps: with the softmax
-// arithmetic switched off (timing-only copy) a key-block still took 3200 cycles
-// against 2048 of tensor work, 3750 with it.  So everything the issuing warp
-// does per key-block is kept short: every shared-memory descriptor and barrier
+// What bounds the kernel: three things within a tenth of one another.  The issuing
+// warp: the tensor pipe accepts an MMA only a couple of instructions ahead, and the
+// issuing thread needs about twenty dependent instructions per tcgen05.mma
+// (election, moves into uniform registers), on a scheduler it shares with two
+// softmax warps; with the softmax arithmetic switched off (timing-only copy) a
+// key-block still takes 3200 cycles against 2048 of tensor work, 3500 with it.
+// Each tile's chain: S ready -> softmax -> P -> its sixteen MMAs -> S ready, 3400
+// cycles, and TMEM holds two tiles.  The schedulers: each hosts one softmax warp of
+// each tile, 2800 cycles of arithmetic per key-block.  So everything the issuing
+// warp does per key-block is kept short: every shared-memory descriptor and barrier
 // address is a compile-time constant (dynamic shared memory starts at offset
 // 0x400 of the CTA's window and a whole-TMEM allocation at column 0; both are
 // checked at kernel start, and the loop is unrolled over the two ring stages so
