@@ -262,12 +262,14 @@ int sp_prefill_attn(sp_ctx* ctx, const sp_tensor* q, const sp_tensor* k, const s
 
 /*
  * The whole layer with HOST buffers: the same steps as sp_prefill_attn (same
- * algorithms of the paper), with the transfers pipelined around them.  The K and V
- * of the pivots' KV heads and the pivots' queries are copied in first, then the
- * other KV heads; the pivots' dense attention and the
- * mask construction run while the members' queries are still arriving; the
- * members run in groups of four heads, each group's outputs copied back while
- * the next group computes.  Copies use two streams owned by the context; when the
+ * algorithms of the paper), with the transfers pipelined around them, cluster by
+ * cluster with the pivots one cluster ahead: pivot 0, pivot 1, the members of
+ * cluster 0, pivot 2, the members of cluster 1, and so on.  A pivot's KV head and
+ * queries are copied in, its dense attention and mask construction run, its
+ * output is copied back; members follow in groups of one or two heads (their KV
+ * head, if it is not on the device yet, and their queries in; attention; output
+ * back) while the next bytes arrive.  Heads of clusters without a pivot run
+ * dense, first.  Copies use two streams owned by the context; when the
  * call returns everything is enqueued, and `stream` is made to wait for the last
  * copy, so synchronising `stream` is enough before reading out_host.  The same
  * holds when the call fails part-way: whatever copies it had already enqueued
