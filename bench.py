@@ -263,6 +263,15 @@ def workload_cfg(args):
     return synth.scaled(cfg, args.seq) if args.seq else cfg
 
 
+def config_dict(cfg, gamma, n_pivots, seed, by_cluster):
+    """The `config` object of the JSON line: the same for both arms (the reference arm runs on this arm's config)."""
+    return {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+            "head_dim": cfg.head_dim, "block": cfg.block, "gamma": gamma, "n_pivots": n_pivots, "seed": seed,
+            "l2": "inputs (2.5 GiB at 128K) exceed the 126 MB L2; no flush between steps",
+            "units_per_rank": ("one layer split by cluster over the ranks (K/V replicated, outputs disjoint, no "
+                               "collective)" if by_cluster else "one layer per rank, independent seeds")}
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
@@ -283,8 +292,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
-                   "head_dim": cfg.head_dim, "block": cfg.block, "gamma": args.gamma, "seed": args.seed},
+        "config": config_dict(cfg, args.gamma, len(L["pivot_heads"]), args.seed, args.shard == "cluster" and world > 1),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -676,11 +684,7 @@ def run_ours(args):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if by_cluster else "weak", "vs_baseline": None,
         "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": cfg.name, "seq": cfg.seq, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
-                   "head_dim": cfg.head_dim, "block": cfg.block, "gamma": gamma, "n_pivots": len(piv),
-                   "seed": args.seed, "l2": "inputs (2.5 GiB at 128K) exceed the 126 MB L2; no flush between steps",
-                   "units_per_rank": ("one layer split by cluster over the ranks (K/V replicated, outputs disjoint, no "
-                                      "collective)" if by_cluster else "one layer per rank, independent seeds")},
+        "config": config_dict(cfg, gamma, len(piv), args.seed, by_cluster),
         "ms_per_layer": ms,
         "kernels_ms": {"pivot_dense_attn": k1, "block_mask": k2, "block_sparse_attn": k3},
         "visited_tiles": {"pivot": pivot_tiles, "members": member_tiles, "causal_per_head": tiles_causal},

@@ -62,6 +62,11 @@ def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
     assert d["impl"] == "reference" and d["metric"] == bench.METRIC and d["unit"] == bench.UNIT
     assert d["value"] > 0 and d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["vs_baseline"] is None
+    # the reference arm runs on the GPU arm's config: one function writes the object for both
+    from paper_2505_19578_b200 import synth
+    cfg = synth.CONFIGS["tiny"]
+    n_piv = len(synth.make_cluster_map(cfg, 0)[1])
+    assert d["config"] == bench.config_dict(cfg, 0.9, n_piv, 0, False)
     env1 = dict(os.environ, RANK="1", WORLD_SIZE="2")
     out1 = subprocess.run(cmd, capture_output=True, text=True, env=env1, timeout=600)
     assert out1.returncode == 0 and out1.stdout.strip() == ""
