@@ -40,6 +40,18 @@ int sp_ctx_set_kernel(sp_ctx* ctx, int which);
  * switches tracing off. */
 int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role);
 
+/* Work order of a launch of the paired attention kernel (head_dim 128, block
+ * 128), computed on the host exactly as the launcher does and walked exactly
+ * as the kernel walks it: for every position raw = 0 .. n_heads *
+ * ceil(n_row_blocks / 2) - 1 the two tiles of the work item,
+ * tiles_out[4 raw ..] = {slot of tile A, row-block of tile A, slot of tile B,
+ * row-block of tile B} (slots index `heads` / `lists`; a row-block >=
+ * n_row_blocks means that the tile does not exist).  n_sm: SM count the launch
+ * is sized for; pair_heads: as kernel selection 0 (non-zero) or 3 (zero).  Host
+ * pointers; no device is touched.  For tests of the order. */
+int sp_internal_pair_work_order(const int32_t* heads, const int32_t* lists, int n_heads, int n_q_heads, int n_kv_heads,
+                                int n_row_blocks, int n_sm, int pair_heads, int32_t* tiles_out, int* n_groups_out);
+
 /* Number of kernels this context has launched since creation (for callers
  * that account for launches). */
 int64_t sp_ctx_launch_count(const sp_ctx* ctx);

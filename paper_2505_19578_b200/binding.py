@@ -36,6 +36,7 @@ EXPORTS = (
     "sp_determine_pattern", "sp_vertical_slash_pattern", "sp_prefill_attn_auto",
     "sp_dict_create", "sp_dict_destroy", "sp_dict_clear", "sp_dict_count", "sp_prefill_attn_layer",
     "sp_selftest_wait_timeout", "sp_fixed_scratch_status", "sp_workspace_bytes_patterns",
+    "sp_internal_pair_work_order",
 )
 
 
@@ -329,6 +330,19 @@ def workspace_bytes_patterns(seq, n_q_heads, n_kv_heads, head_dim, block, n_pivo
                                               int(bool(pooled_construction)), ctypes.byref(a), ctypes.byref(b)),
            "sp_workspace_bytes_patterns")
     return a.value, b.value
+
+
+def pair_work_order(heads, lists, n_q_heads, n_kv_heads, n_row_blocks, n_sm=148, pair_heads=True):
+    """Work order of a paired-kernel launch, computed on the host: (items, n_groups), items[raw] = (slot of tile A,
+    row-block of tile A, slot of tile B, row-block of tile B).  Touches no device."""
+    heads, lists = list(heads), list(lists)
+    n_items = len(heads) * ((n_row_blocks + 1) // 2)
+    tiles = (ctypes.c_int32 * (4 * n_items))()
+    ng = ctypes.c_int()
+    _check(load().sp_internal_pair_work_order(_i32(heads), _i32(lists), len(heads), n_q_heads, n_kv_heads, n_row_blocks,
+                                              n_sm, int(bool(pair_heads)), tiles, ctypes.byref(ng)),
+           "sp_internal_pair_work_order")
+    return [tuple(tiles[4 * r:4 * r + 4]) for r in range(n_items)], ng.value
 
 
 def fixed_scratch_status(device=0):

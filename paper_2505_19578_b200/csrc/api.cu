@@ -343,6 +343,31 @@ int sp_ctx_set_kernel(sp_ctx* ctx, int which) {
 
 int64_t sp_ctx_launch_count(const sp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int sp_internal_pair_work_order(const int32_t* heads, const int32_t* lists, int n_heads, int n_q_heads, int n_kv_heads,
+                                int n_row_blocks, int n_sm, int pair_heads, int32_t* tiles_out, int* n_groups_out) {
+  if (!heads || !lists || !tiles_out || n_heads <= 0 || n_heads > kMaxHeads || n_q_heads <= 0 || n_kv_heads <= 0 ||
+      n_q_heads % n_kv_heads != 0 || n_row_blocks <= 0 || n_sm <= 0)
+    return SP_ERR_INVALID_ARG;
+  AttnArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n_heads = n_heads; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.group = n_q_heads / n_kv_heads;
+  a.Nb = n_row_blocks; a.pair_heads = pair_heads;
+  for (int t = 0; t < n_heads; ++t) {
+    if (heads[t] < 0 || heads[t] >= n_q_heads) return SP_ERR_INVALID_ARG;
+    a.heads.v[t] = heads[t];
+    a.lists.v[t] = lists[t];
+  }
+  attn_pair_work_order(a, n_sm);
+  const int n_items = n_heads * ((n_row_blocks + 1) / 2);
+  for (int raw = 0; raw < n_items; ++raw) {
+    int sa, ra, sb, rb;
+    if (!attn_pair_item(a, raw, &sa, &ra, &sb, &rb)) return SP_ERR_INVALID_ARG;
+    tiles_out[4 * raw + 0] = sa; tiles_out[4 * raw + 1] = ra; tiles_out[4 * raw + 2] = sb; tiles_out[4 * raw + 3] = rb;
+  }
+  if (n_groups_out) *n_groups_out = a.n_groups;
+  return SP_OK;
+}
+
 int sp_ctx_set_trace(sp_ctx* ctx, int64_t* events, int events_per_role) {
   if (!ctx || events_per_role < 0 || (events_per_role > 0 && !events)) return SP_ERR_INVALID_ARG;
   ctx->trace = events_per_role > 0 ? reinterpret_cast<long long*>(events) : nullptr;

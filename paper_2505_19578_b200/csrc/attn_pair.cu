@@ -275,6 +275,27 @@ enum { ITEM_INTS = 16 };
 // one KV head that walk the same list (tile A = row-block i of the first, tile B = row-block i of the second; one entry
 // for the even i, one for the odd i, so that every entry has ceil(Nb / 2) items).
 enum { ENT_ONE_HEAD = 0, ENT_TWO_HEADS_EVEN = 1, ENT_TWO_HEADS_ODD = 2 };
+// Position `raw` of the work order -> its two tiles.  Groups in turn; inside a group the longest pairs first, entries
+// fastest.
+struct WorkItemTiles { int slot_a, slot_b, rb_a, rb_b; };
+__host__ __device__ inline WorkItemTiles resolve_item(const HeadTable& order, const GroupTable& group_start, int n_groups,
+                                                      int n_pairs, int raw) {
+  int rest = raw, g = 0;
+  while (g + 1 < n_groups && rest >= (group_start.v[g + 1] - group_start.v[g]) * n_pairs) {
+    rest -= (group_start.v[g + 1] - group_start.v[g]) * n_pairs;
+    ++g;
+  }
+  const int ng = group_start.v[g + 1] - group_start.v[g];
+  const int ent = order.v[group_start.v[g] + rest % ng];
+  const int u = n_pairs - 1 - rest / ng;
+  const int kind = ent >> 16;
+  WorkItemTiles w;
+  w.slot_a = ent & 0xff;
+  w.slot_b = (ent >> 8) & 0xff;
+  w.rb_a = kind == ENT_ONE_HEAD ? 2 * u : 2 * u + (kind - ENT_TWO_HEADS_EVEN);
+  w.rb_b = kind == ENT_ONE_HEAD ? 2 * u + 1 : w.rb_a;
+  return w;
+}
 
 // Rare path of the softmax, kept out of the hot loop: the row's reference max has moved, so O of the earlier
 // steps (when there are any) and the P chunks of this key-block that are already stored are brought to the new
@@ -413,20 +434,12 @@ attn_pair_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap tm_q, con
           if (lane == 0) {
             const int raw = poisoned ? n_items : atomicAdd(a.work_counter, 1);
             if (raw < n_items) {
-              int rest = raw, g = 0;
-              while (g + 1 < a.n_groups && rest >= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs) {
-                rest -= (a.group_start.v[g + 1] - a.group_start.v[g]) * n_pairs;
-                ++g;
-              }
-              const int ng = a.group_start.v[g + 1] - a.group_start.v[g];
-              const int ent = a.order.v[a.group_start.v[g] + rest % ng];
-              const int u = n_pairs - 1 - rest / ng;
-              const int kind = ent >> 16;
+              const WorkItemTiles w = resolve_item(a.order, a.group_start, a.n_groups, n_pairs, raw);
               it.id = raw;
-              it.slotA = sp_in_range(ent & 0xff, 0, a.n_heads - 1, a.status, 51);
-              it.slotB = sp_in_range((ent >> 8) & 0xff, 0, a.n_heads - 1, a.status, 51);
-              it.iA = kind == ENT_ONE_HEAD ? 2 * u : 2 * u + (kind - ENT_TWO_HEADS_EVEN);
-              it.iB = kind == ENT_ONE_HEAD ? 2 * u + 1 : it.iA;
+              it.slotA = sp_in_range(w.slot_a, 0, a.n_heads - 1, a.status, 51);
+              it.slotB = sp_in_range(w.slot_b, 0, a.n_heads - 1, a.status, 51);
+              it.iA = w.rb_a;
+              it.iB = w.rb_b;
               it.hA = sp_in_range(a.heads.v[it.slotA], 0, a.n_q_heads - 1, a.status, 51);
               it.hB = sp_in_range(a.heads.v[it.slotB], 0, a.n_q_heads - 1, a.status, 51);
               it.listA = a.lists_dev ? a.lists_dev[it.slotA] : a.lists.v[it.slotA];
@@ -885,18 +898,15 @@ size_t attn_pair_stats_bytes(int n_heads, int Nb) {
   return (size_t)attn_pair_ctas(n_heads, Nb) * 2 * (size_t)Nb * BLK * sizeof(float);
 }
 
-cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
-  if (!attn_pair_supported(a_in) || !a_in.work_counter) return cudaErrorInvalidValue;
-  AttnArgs a = a_in;
-  // Work order.  Many items (forty per SM or more): the slots sorted by KV head (stable), one group per KV head,
-  // so that a K/V set stays in L2 while its heads run.  Fewer: one group, i.e. the longest pairs of all heads
-  // first, because then the balance at the end matters more than L2.
-  // Two heads of one KV head that walk the same list (members of one cluster; two dense heads) share a work item
-  // row-block by row-block: their two tiles need exactly the same K/V tiles, so no K/V load serves one tile alone,
-  // as happens wherever two adjacent row-blocks of one head differ in their lists.  Such a pair takes two entries
-  // (even and odd row-blocks); a head without a partner keeps one entry and pairs its own adjacent row-blocks.
-  // Lists decided on the device are not known here: those heads stay single.
-  const int n_sm = sm_count();
+// Work order of a launch (host).  Many items (forty per SM or more): the slots sorted by KV head (stable), one group
+// per KV head, so that a K/V set stays in L2 while its heads run.  Fewer: one group, i.e. the longest pairs of all
+// heads first, because then the balance at the end matters more than L2.
+// Two heads of one KV head that walk the same list (members of one cluster; two dense heads) share a work item
+// row-block by row-block: their two tiles need exactly the same K/V tiles, so no K/V load serves one tile alone,
+// as happens wherever two adjacent row-blocks of one head differ in their lists.  Such a pair takes two entries
+// (even and odd row-blocks); a head without a partner keeps one entry and pairs its own adjacent row-blocks.
+// Lists decided on the device are not known here: those heads stay single.
+void attn_pair_work_order(AttnArgs& a, int n_sm) {
   const bool by_kv_head = (long)a.n_heads * ((a.Nb + 1) / 2) >= 40L * n_sm;
   int n = 0;
   a.n_groups = 0;
@@ -935,6 +945,22 @@ cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
   static_assert(kMaxHeads <= 256, "an entry of the work order holds two slots of eight bits");
   static_assert(sizeof(a.group_start.v) / sizeof(a.group_start.v[0]) == kMaxHeads + 1, "room for the end of the last group");
   a.group_start.v[a.n_groups] = n;
+}
+
+// Position `raw` of the work order -> the two tiles (slot and row-block of each); what the producer warp does on the
+// device, here for host-side checks of the order.  False past the end.
+bool attn_pair_item(const AttnArgs& a, int raw, int* slot_a, int* rb_a, int* slot_b, int* rb_b) {
+  const int n_pairs = (a.Nb + 1) / 2;
+  if (raw < 0 || raw >= a.n_heads * n_pairs) return false;
+  WorkItemTiles w = resolve_item(a.order, a.group_start, a.n_groups, n_pairs, raw);
+  *slot_a = w.slot_a; *rb_a = w.rb_a; *slot_b = w.slot_b; *rb_b = w.rb_b;
+  return true;
+}
+
+cudaError_t launch_attn_pair(const AttnArgs& a_in, cudaStream_t s) {
+  if (!attn_pair_supported(a_in) || !a_in.work_counter) return cudaErrorInvalidValue;
+  AttnArgs a = a_in;
+  attn_pair_work_order(a, sm_count());
   CUtensorMap tq, tk, tv;
   if (!make_map(&tq, a.q, a.q_sh, a.q_sn, a.n_q_heads, a.N, D, BLK) ||
       !make_map(&tk, a.k, a.k_sh, a.k_sn, a.n_kv_heads, a.N, D, BLK) ||

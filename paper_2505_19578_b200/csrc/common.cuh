@@ -115,6 +115,9 @@ cudaError_t launch_attn_pair(const AttnArgs& a, cudaStream_t s);
 // CTAs a paired launch over n_heads heads runs (one per SM of the current device at most), and the bytes of
 // tile statistics it needs when it emits importance: one region of 2 * Nb * 128 floats per CTA
 int attn_pair_ctas(int n_heads, int Nb);
+// host: the work order of a paired launch (fills order, group_start, n_groups), and position -> its two tiles
+void attn_pair_work_order(AttnArgs& a, int n_sm);
+bool attn_pair_item(const AttnArgs& a, int raw, int* slot_a, int* rb_a, int* slot_b, int* rb_b);
 size_t attn_pair_stats_bytes(int n_heads, int Nb);
 // dense attention with importance, statistics, status word and work counter in the library's fixed device arrays
 // (the paired kernel at head_dim 128 / block 128, the one-row-block kernel otherwise)

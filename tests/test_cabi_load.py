@@ -65,3 +65,58 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.load()
+
+
+def test_work_order_of_the_paired_kernel_covers_every_tile_once(lib):
+    """Host logic of a paired-kernel launch: every (head, row-block) is one tile of exactly one work item; two heads
+    share items only if they read the same KV head and walk the same list; a launch of many items keeps the heads of
+    a KV head together and, inside such a group, the long row-blocks first."""
+    import random
+    from paper_2505_19578_b200 import binding
+    rnd = random.Random(11)
+    cases = [([4, 0, 3, 5, 1, 2], [1, 0, 1, -1, 1, -1], 6, 1, 11, 148)]            # the GPU test's case: 2 pairs + 2 single
+    for _ in range(60):
+        hkv = rnd.choice([1, 2, 4, 8])
+        hq = hkv * rnd.choice([1, 2, 4, 7])
+        n_heads = rnd.randint(1, hq)
+        heads = rnd.sample(range(hq), n_heads)
+        lists = [rnd.choice([-1, 0, 1, 2]) for _ in heads]
+        cases.append((heads, lists, hq, hkv, rnd.choice([1, 2, 3, 8, 9, 64, 257]), rnd.choice([4, 148])))
+    for heads, lists, hq, hkv, nb, n_sm in cases:
+        group = hq // hkv
+        for pair_heads in (True, False):
+            items, n_groups = binding.pair_work_order(heads, lists, hq, hkv, nb, n_sm, pair_heads)
+            assert len(items) == len(heads) * ((nb + 1) // 2)
+            seen = {}
+            for raw, (sa, ra, sb, rb) in enumerate(items):
+                assert 0 <= sa < len(heads) and 0 <= sb < len(heads) and ra >= 0 and rb >= 0
+                assert heads[sa] // group == heads[sb] // group                   # one K/V stream per item
+                if sa != sb:
+                    assert pair_heads and ra == rb                                # two heads: the same row-block,
+                    assert max(lists[sa], -1) == max(lists[sb], -1)               # ... the same list
+                else:
+                    assert rb == ra + 1 and ra % 2 == 0                           # one head: adjacent row-blocks
+                for s_, r_ in ((sa, ra), (sb, rb)):
+                    if r_ < nb:
+                        assert (s_, r_) not in seen, (heads, lists, nb, raw)
+                        seen[(s_, r_)] = raw
+            assert len(seen) == len(heads) * nb                                   # every tile, once
+            by_kv = len(heads) * ((nb + 1) // 2) >= 40 * n_sm
+            assert n_groups == (len({h // group for h in heads}) if by_kv else 1)
+            # the heads of a KV head stay together (many items), and inside a group the pairs of row-blocks never grow
+            last_u, last_kv, closed = None, None, set()
+            for sa, ra, sb, rb in items:
+                kv = heads[sa] // group
+                if by_kv and kv != last_kv:
+                    assert kv not in closed
+                    closed.add(kv)
+                    last_kv, last_u = kv, None
+                assert last_u is None or ra // 2 <= last_u
+                last_u = ra // 2
+    # the 128K workload: 16 of the 28 members find a partner
+    from paper_2505_19578_b200 import synth
+    cfg = synth.CONFIGS["llama8b_128k"]
+    cm, piv = synth.make_cluster_map(cfg, 0)
+    members = [h for h in range(cfg.n_q_heads) if h not in piv]
+    items, _ = binding.pair_work_order(members, [cm[h] for h in members], cfg.n_q_heads, cfg.n_kv_heads, 1024)
+    assert len({s for sa, _, sb, _ in items if sa != sb for s in (sa, sb)}) == 16
