@@ -489,7 +489,7 @@ def run_ours(args):
     # ---- the other configurations named next to the default one: the gamma sweep on the same inputs, the 32K and the
     #      GQA-7 64K layer (a few steps each; per-kernel times, visited-tile rates, dense, clocks)
     others = None
-    if rank == 0 and not args.no_other_configs and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9:
+    if world == 1 and not args.no_other_configs and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9:
         others = []
         n_other = max(2, min(args.steps, 5))
         for g_ in (0.8, 0.95):
@@ -505,7 +505,7 @@ def run_ours(args):
     #      sp_prefill_attn_auto, then a stack of layers through the cross-layer dictionary (pivots only where a cluster
     #      has no pattern yet; later layers reuse what earlier ones stored)
     mixed = None
-    if (rank == 0 and not args.no_mixed and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9):
+    if (world == 1 and not args.no_mixed and not args.seq and args.workload == "llama8b_128k" and gamma == 0.9):
         mcfg = synth.CONFIGS["llama8b_128k_mixed"]
         Lm = synth.make_layer(mcfg, seed=args.seed, device=str(dev))
         mout = torch.empty_like(Lm["q"])
@@ -560,7 +560,7 @@ def run_ours(args):
 
     # ---- the paper-literal construction beside it (block-averaged QK values, global cut): time and what it selects
     literal = None
-    if rank == 0 and not args.no_literal:
+    if world == 1 and not args.no_literal:      # (with several ranks the other GPUs would only stand by)
         pooled = torch.empty(len(piv), Nb, Nb, dtype=torch.float64, device=dev)
         lm = torch.empty(len(piv), Nb, Nb, dtype=torch.uint8, device=dev)
         lc = torch.empty(len(piv), Nb, dtype=torch.int32, device=dev)
