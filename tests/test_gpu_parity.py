@@ -427,3 +427,66 @@ def test_random_small_shapes_tensor_core_path_agrees_with_cuda_core_path(binding
         assert not torch.isnan(res["tc"][0]).any(), (case, nb, hq, piv, gamma)
         assert torch.equal(res["tc"][1], res["simt"][1]), (case, nb, hq, piv, gamma)
         assert (res["tc"][0] - res["simt"][0]).abs().max().item() < 2e-2, (case, nb, hq, piv, gamma)
+
+
+def test_random_lists_heads_and_host_call(binding):
+    """Random head subsets, list assignments (repeated lists on one KV head: shared work items; dense heads; several
+    lists), densities and lengths: the block-sparse call with two heads per work item is bit-identical to one head per
+    item and agrees with the CUDA-core kernel; the host-buffer call of the whole layer is bit-identical to the
+    device-pointer call.  (Oracle parity of the same calls is covered above at fixed shapes.)"""
+    import dataclasses
+    import random
+    rnd = random.Random(23)
+    ctxs = {kern: binding.Context(kernel=kern) for kern in ("tc", "tc_single_head_items", "simt")}
+    base = synth.CONFIGS["llama8b_32k"]
+    for case in range(40):
+        nb = rnd.choice([1, 2, 3, 5, 8, 9, 17, 33])
+        hkv = rnd.choice([1, 2, 4])
+        hq = hkv * rnd.choice([1, 2, 4, 8])
+        cfg = dataclasses.replace(base, seq=nb * 128, n_q_heads=hq, n_kv_heads=hkv, n_clusters=rnd.randint(1, min(4, hq)),
+                                  n_heavy=min(base.n_heavy, nb * 128 - 2), name="random")
+        L = synth.make_layer(cfg, seed=500 + case, device="cuda")
+        q, k, v = L["q"], L["k"], L["v"]
+        g = np.random.default_rng(case)
+        n_lists = rnd.randint(1, 3)
+        dens = rnd.choice([0.1, 0.3, 0.6, 1.0])
+        masks = np.zeros((n_lists, nb, nb), np.uint8)
+        for l in range(n_lists):
+            m = np.tril(g.random((nb, nb)) < dens).astype(np.uint8)
+            for i in range(nb):
+                if m[i].sum() == 0:
+                    m[i, g.integers(0, i + 1)] = 1
+            masks[l] = m
+        counts = torch.from_numpy(masks.sum(axis=2).astype(np.int32)).cuda()
+        idx = np.full((n_lists, nb, nb), -1, np.int32)
+        for l in range(n_lists):
+            for i in range(nb):
+                sel = np.nonzero(masks[l, i])[0]
+                idx[l, i, :len(sel)] = sel
+        idx = torch.from_numpy(idx).cuda()
+        heads = rnd.sample(range(hq), rnd.randint(1, hq))
+        lists = [rnd.choice([-1] + list(range(n_lists))) for _ in heads]
+        outs = {}
+        for kern, ctx in ctxs.items():
+            out = torch.zeros_like(q)
+            ctx.sp_block_sparse_attn(q, k, v, heads, lists, counts, idx, cfg.block, out)
+            _sync_ok(ctx)
+            outs[kern] = out
+        what = (case, nb, hq, hkv, heads, lists)
+        assert torch.equal(outs["tc"], outs["tc_single_head_items"]), what
+        assert (outs["tc"].float() - outs["simt"].float()).abs().max().item() < 2e-2, what
+        cm, piv = list(L["cluster_map"]), list(L["pivot_heads"])
+        if rnd.random() < 0.3 and len(piv) > 1:
+            piv = piv[:-1]
+        if rnd.random() < 0.3:
+            cm[rnd.randrange(hq)] = -1
+        gamma = rnd.choice([0.5, 0.9, 0.99])
+        ctx = ctxs["tc"]
+        o_dev = torch.zeros_like(q)
+        ctx.sp_prefill_attn(q, k, v, cm, piv, gamma, cfg.block, o_dev)
+        _sync_ok(ctx)
+        ho = torch.zeros(q.shape, dtype=q.dtype).pin_memory()
+        ctx.sp_prefill_attn_host(q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory(), cm, piv, gamma,
+                                 cfg.block, ho)
+        _sync_ok(ctx)
+        assert torch.equal(ho, o_dev.cpu()), what
